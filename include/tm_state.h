@@ -1,0 +1,183 @@
+/*
+ * tm_state.h — C ABI of the role-state mover.
+ *
+ * The operation family implemented here is the bulk state hand-over that
+ * TrainMover performs in its switching phase (paper §7 "Implementation",
+ * paragraph "State Synchronization"): a leaver sends its latest training
+ * state — model parameters and optimizer states — to the joiner that takes
+ * over its role, and with a distributed (ZeRO-style) optimizer a joiner needs
+ * the slice of the optimizer state that belongs to its data-parallel rank.
+ * §8.5 "Zero Memory Overhead Workflow" adds that the state travels through a
+ * staging channel (the leaver's recycled gradient buffer), which is why the
+ * state is first packed into flat, fixed-size transfer buckets.  The paper
+ * fixes no wire format; the format below (256-byte alignment, fixed-size
+ * buckets, floor shard bounds, weighted 64-bit word checksum) is this
+ * library's definition.
+ *
+ * Definitions (all arithmetic on byte offsets is exact, uint64):
+ *
+ *   align256(x)   = (x + 255) & ~255
+ *   Packed stream : descriptors are taken in the order given (never sorted).
+ *                   off_0 = 0, off_k = align256(off_{k-1} + nbytes_{k-1}),
+ *                   T = align256(off_last + nbytes_last).  Stream byte
+ *                   off_k + j is byte j of tensor k; every other byte of
+ *                   [0, T) is 0x00.
+ *   Buckets       : bucket_bytes = B, a positive multiple of 256.  Bucket j is
+ *                   stream bytes [j*B, min((j+1)*B, T)); n_buckets =
+ *                   ceil(T / B).  Tensors may straddle buckets.  The packed
+ *                   buffer is the contiguous stream, bucket j at byte j*B.
+ *   Checksum      : for a bucket of L bytes, n = ceil(L / 8) little-endian
+ *                   uint64 words w_i (missing bytes read as zero);
+ *                   C = sum_{i=0}^{n-1} w_i * (2*i + 1)  mod 2^64.
+ *                   i restarts at 0 in every bucket.
+ *   Shard         : a plane is an ordered list of tensors with one common
+ *                   elem_size e, viewed as one flat array of N elements
+ *                   (concatenated WITHOUT padding).  The shard of data-parallel
+ *                   rank r of D is elements [floor(r*N/D), floor((r+1)*N/D)),
+ *                   written contiguously.  The products are formed in 128 bits.
+ *
+ * Conventions
+ *   - Every pointer whose name starts with d_ is a DEVICE pointer; tm_desc.ptr
+ *     is a device pointer; everything else is a HOST pointer.
+ *   - The caller owns all device memory (tensors, packed buffer, checksum
+ *     array, workspace) and the stream.  The library allocates no device
+ *     memory.  A tm_plan owns host memory only, plus the contents it wrote
+ *     into the workspace handed to tm_plan_upload.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  All device work is enqueued on it and the call returns without
+ *     waiting; the caller synchronises.  The device of the stream/pointers must
+ *     be the current device.
+ *   - Every argument is validated on the host before anything is launched.
+ *     Functions return TM_OK (0) or a negative tm_status.  On error nothing has
+ *     been enqueued.  There is no CPU fallback: without a usable CUDA device
+ *     the operations return TM_ERR_CUDA.
+ *   - Tensor addresses need only 2-byte alignment.  To serve such tensors at
+ *     full speed the kernels read whole 16-byte-aligned lines: a line that
+ *     holds at least one byte of a tensor may be read in full (it lies in the
+ *     same memory page as that byte), but bytes outside the tensor are never
+ *     used and never written.
+ */
+#ifndef TM_STATE_H
+#define TM_STATE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum tm_status {
+  TM_OK           =  0,
+  TM_ERR_ARG      = -1,  /* NULL pointer, zero count/size, odd nbytes, nbytes % elem_size != 0 */
+  TM_ERR_ALIGN    = -2,  /* odd tensor address, bucket_bytes % 256 != 0, packed buffer not 256-byte aligned */
+  TM_ERR_CAPACITY = -3,  /* output, input or workspace buffer smaller than required */
+  TM_ERR_OVERLAP  = -4,  /* a tensor overlaps the packed/output buffer, or two unpack targets overlap */
+  TM_ERR_RANK     = -5,  /* D == 0 or r >= D */
+  TM_ERR_DTYPE    = -6,  /* elem_size not in {2,4,8}, or mixed elem_size inside one shard plane */
+  TM_ERR_CUDA     = -7,  /* a CUDA runtime call failed (tm_last_cuda_error() gives its code) */
+  TM_ERR_TIMEOUT  = -8,  /* a bounded device-side wait expired (reported by tm_plan_status / tm_workspace_status) */
+  TM_ERR_STATE    = -9   /* the plan has no uploaded work list (tm_plan_upload not called) */
+} tm_status;
+
+/* One tensor of a role's training state. */
+typedef struct tm_desc {
+  void*    ptr;        /* device address, >= 2-byte aligned; source for pack and shard, destination for unpack */
+  uint64_t nbytes;     /* numel * elem_size; > 0 */
+  uint32_t elem_size;  /* 2 (bf16), 4 (fp32) or 8 (int64) */
+  uint32_t plane;      /* caller's label: 0 bf16 param, 1 fp32 master, 2 Adam m, 3 Adam v, 4 other; not interpreted */
+} tm_desc;
+
+typedef struct tm_plan tm_plan;  /* opaque */
+
+/* ---- plan: layout of a role's tensors in the packed stream ------------------------------- */
+
+/* Computes the packed-stream layout (off_k, T, buckets; definitions above) for `n_desc`
+ * descriptors and cuts it into the device work list.  Host only: no CUDA call is made.
+ * `descs` is copied; it may be freed after the call.  *out receives a plan to be released with
+ * tm_plan_destroy.  Errors: TM_ERR_ARG (NULL, n_desc == 0, nbytes == 0, nbytes % elem_size != 0,
+ * bucket_bytes == 0 or > 2^35), TM_ERR_DTYPE, TM_ERR_ALIGN (odd ptr, bucket_bytes % 256 != 0). */
+int tm_plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_plan** out);
+
+/* Any of the three outputs may be NULL.  total_bytes = T, n_buckets = ceil(T/B),
+ * workspace_bytes = size the caller must provide to tm_plan_upload. */
+int tm_plan_query(const tm_plan* plan, uint64_t* total_bytes, uint64_t* n_buckets,
+                  uint64_t* workspace_bytes);
+
+/* Writes off_k for every descriptor into host array `offsets` (n_desc entries). */
+int tm_plan_offsets(const tm_plan* plan, uint64_t* offsets);
+
+/* Copies the work list into caller-owned device memory `d_workspace` (256-byte aligned, at
+ * least workspace_bytes from tm_plan_query) on `stream`.  The workspace must stay untouched
+ * while the plan is in use.  Calling it again re-targets the plan to another workspace. */
+int tm_plan_upload(tm_plan* plan, void* d_workspace, uint64_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, then reads the plan's device status word: *device_status = TM_OK, or
+ * TM_ERR_TIMEOUT if any kernel launched with this plan gave up a bounded wait (its output is
+ * then incomplete).  Returns TM_ERR_CUDA if the synchronisation itself failed. */
+int tm_plan_status(const tm_plan* plan, void* stream, int* device_status);
+
+void tm_plan_destroy(tm_plan* plan);
+
+/* ---- the four operations ------------------------------------------------------------------- */
+
+/* Pack (leaver side of "State Synchronization", §7; bucket staging per §8.5).
+ * Gathers every tensor of the plan into d_buckets[0, T) following the packed-stream definition,
+ * writes all padding bytes as zero, and — in the same pass over the data — accumulates the
+ * checksum of each bucket.  d_buckets: device, 256-byte aligned, `capacity` >= T bytes, must not
+ * overlap any tensor.  d_checksums: device array of n_buckets uint64 (8-byte aligned) that
+ * receives the checksums, or NULL to skip them.  Enqueues on `stream`. */
+int tm_state_pack(const tm_plan* plan, void* d_buckets, uint64_t capacity,
+                  uint64_t* d_checksums, void* stream);
+
+/* Unpack (joiner side: the received state overwrites the sandbox-warmed state, §7 and §4.2).
+ * Copies nbytes_k bytes from d_buckets + off_k into tensor k for every k; padding is ignored.
+ * `nbytes` = valid bytes at d_buckets, must be >= T.  d_buckets 256-byte aligned.  The tensors
+ * must not overlap the packed buffer or one another. */
+int tm_state_unpack(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, void* stream);
+
+/* Host helper: floor shard bounds lo = floor(r*N/D), hi = floor((r+1)*N/D) in 128-bit arithmetic. */
+int tm_shard_bounds(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
+
+/* Workspace size tm_shard_extract needs for a plane of n_desc tensors and the given bounds.
+ * Returns the size in *workspace_bytes. */
+int tm_shard_workspace(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                       uint64_t* workspace_bytes);
+
+/* Shard extract (state for a joiner under the distributed optimizer, §7 "State
+ * Synchronization": no replica holds the shard, so it is cut out of the flat plane).
+ * plane_descs: host array of n_desc tensors with one common elem_size (TM_ERR_DTYPE otherwise),
+ * viewed as one flat array without padding.  Copies elements [lo, hi) (definition above) to
+ * d_out (device, >= 2-byte aligned, out_capacity bytes >= (hi-lo)*elem_size, no overlap with the
+ * tensors).  *out_elems (host, may be NULL) receives hi - lo, which may be 0 (nothing is then
+ * launched).  d_workspace: caller-owned device scratch, 256-byte aligned, at least
+ * tm_shard_workspace() bytes; it must stay untouched until the enqueued work has finished.
+ * Errors: TM_ERR_RANK for D == 0 or r >= D. */
+int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                     void* d_out, uint64_t out_capacity, uint64_t* out_elems,
+                     void* d_workspace, uint64_t workspace_bytes, void* stream);
+
+/* Status word of a raw workspace used by tm_shard_extract (same meaning as tm_plan_status). */
+int tm_workspace_status(const void* d_workspace, void* stream, int* device_status);
+
+/* Checksum (integrity check of received buckets; the paper has no integrity check, the formula
+ * is this library's, see "Checksum" above).  Treats d_bytes[0, nbytes) as ceil(nbytes /
+ * bucket_bytes) buckets and writes one uint64 per bucket to d_checksums.  d_bytes must be
+ * 16-byte aligned; nbytes may be any value (the last word is zero-extended); nbytes == 0 writes
+ * nothing.  bucket_bytes: positive multiple of 256, <= 2^35. */
+int tm_checksum(const void* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
+                uint64_t* d_checksums, void* stream);
+
+/* ---- diagnostics ----------------------------------------------------------------------------- */
+
+const char* tm_strerror(int status);
+
+/* cudaError_t value of the most recent failed CUDA runtime call made by this library (0 if none). */
+int tm_last_cuda_error(void);
+
+/* Number of kernels this library has launched since it was loaded (all streams, all threads). */
+uint64_t tm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TM_STATE_H */
