@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Throughput of the role-state hot path: pack (+fused checksum) -> stand-alone checksum ->
+unpack -> distributed-optimizer shard extract (three fp32 planes), on one synthetic role layout.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl ours|reference]
+
+One "step" is one pass of all four operations over the whole role.  The metric is GB/s of
+algorithmic bytes (bytes read + bytes written by the four operations) over device time.  With
+N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the same role
+on its own GPU — the path has no exchange step — and the value is the sum of the ranks' bytes
+over the slowest rank's time.  `--impl reference` times the CPU oracle on a bounded sample of the
+same workload instead.  Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from typing import Dict, List, Optional, Tuple
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+import torch.distributed as dist
+
+METRIC = "role-state pack/unpack+checksum+shard GB/s and % of B200 HBM peak per role"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+WORKLOADS = {"cfg0": 0, "cfg1": 1, "cfg2": 2, "cfg3": 3}
+
+
+# ------------------------------------------------------------------------------------------------
+# pieces that do not need a GPU (also exercised by the CPU tests)
+
+
+def measured_hbm_peak() -> Tuple[float, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def step_bytes(state_bytes: int, total_bytes: int, n_buckets: int, shard_bytes: List[int]) -> Dict[str, int]:
+    """Algorithmic bytes (read + written) of each operation of one step."""
+    return {
+        "pack": state_bytes + total_bytes + 8 * n_buckets,      # read tensors, write stream + checksums
+        "checksum": total_bytes + 8 * n_buckets,                # read stream, write checksums
+        "unpack": state_bytes + state_bytes,                    # read tensor bytes of the stream, write tensors
+        "shard": sum(2 * b for b in shard_bytes),               # read slice, write slice, per plane
+    }
+
+
+def aggregate_over_ranks(elapsed_ms: float, nbytes: int) -> Tuple[float, int]:
+    """(slowest rank's time, bytes moved by all ranks).  Ranks are independent replicas."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return elapsed_ms, nbytes
+    dev = torch.device("cuda", torch.cuda.current_device()) if dist.get_backend() == "nccl" else torch.device("cpu")
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+    b = torch.tensor([nbytes], dtype=torch.int64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(b.item())
+
+
+def gbs(nbytes: float, ms: float) -> float:
+    return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc: Optional[subprocess.Popen] = None
+        self.lines: List[str] = []
+        self.thread: Optional[threading.Thread] = None
+
+    def start(self) -> None:
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        def pump():
+            for line in self.proc.stdout:
+                self.lines.append(line.strip())
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self) -> Dict[str, object]:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        return self.summarise(self.lines)
+
+    @staticmethod
+    def summarise(lines: List[str]) -> Dict[str, object]:
+        mhz, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                mhz.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(mhz), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (the cpu_baseline leg and --impl reference)
+
+
+def oracle_sample_step(cfg, device="cpu"):
+    """Builds the bounded sample — layer 0's tensors (for cfg0: the whole role) in all four planes —
+    on the host and returns a callable that runs the four oracle operations once over it,
+    returning (seconds, algorithmic bytes)."""
+    import numpy as np
+    import oracle
+    from paper_2412_12636_b200 import layouts
+    oracle.build()
+    specs = cfg.specs()
+    if cfg.index == 0:
+        keep = list(range(len(specs)))
+        what = "whole role"
+    else:
+        keep = [i for i, s in enumerate(specs) if ".l0." in s.name]
+        what = "layer 0 of every plane"
+    host = [layouts.tensor_bytes(layouts._fill_model_tensor(cfg, specs[i], torch.device("cpu"))).numpy() for i in keep]
+    sizes = [h.size for h in host]
+    fp32 = {p: [j for j, i in enumerate(keep) if specs[i].plane == p] for p in (1, 2, 3)}
+    state_bytes = sum(sizes)
+    _, total, nb = oracle.layout(sizes, cfg.bucket_bytes)
+    stream = np.empty(total, dtype=np.uint8)
+
+    def step():
+        t0 = time.perf_counter()
+        s, _ = oracle.pack(host, cfg.bucket_bytes, out=stream)
+        oracle.checksum(s, cfg.bucket_bytes)
+        oracle.unpack(s, sizes)
+        shard_bytes = []
+        for p in (1, 2, 3):
+            out = oracle.shard([host[j] for j in fp32[p]], [sizes[j] for j in fp32[p]], 4, cfg.shard_r, cfg.shard_D)
+            shard_bytes.append(out.size)
+        dt = time.perf_counter() - t0
+        return dt, sum(step_bytes(state_bytes, total, nb, shard_bytes).values())
+
+    sample = f"{what}: {len(keep)} tensors, {state_bytes / 1e9:.3f} GB of state, same four operations, shard r={cfg.shard_r} of {cfg.shard_D}"
+    return step, sample
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2412_12636_b200 import layouts
+    cfg = layouts.role_config(WORKLOADS[args.workload])
+    step, sample = oracle_sample_step(cfg)
+    for _ in range(min(args.warmup, 1)):
+        step()
+    times, nbytes = [], 0
+    for _ in range(max(1, args.steps)):
+        dt, nbytes = step()
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = gbs(nbytes, ms)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(times), "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8/u64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}:{cfg.name}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores_available": os.cpu_count()},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA path
+
+
+def run_ours(args) -> None:
+    from paper_2412_12636_b200 import binding, layouts
+    from paper_2412_12636_b200.mover import RoleMover, ShardExtractor
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    binding.load_library()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg = layouts.role_config(WORKLOADS[args.workload])
+    state = layouts.materialize(cfg, "cuda")
+    target = layouts.blank_like(state)
+    mover = RoleMover(state.descs(), cfg.bucket_bytes)
+    unmover = RoleMover(target.descs(), cfg.bucket_bytes)
+    buckets = mover.alloc_buckets()
+    cks_fused = mover.alloc_checksums()
+    cks_alone = mover.alloc_checksums()
+    shards = []
+    for plane in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V):
+        ex = ShardExtractor([target.descs()[i] for i in target.plane_indices(plane)], cfg.shard_r, cfg.shard_D)
+        shards.append((ex, ex.alloc_out()))
+    per_op = step_bytes(state.state_bytes, mover.total_bytes, mover.n_buckets, [ex.out_bytes for ex, _ in shards])
+    bytes_per_step = sum(per_op.values())
+    stream = torch.cuda.current_stream()
+
+    def one_step(events=None):
+        marks = []
+        def mark():
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(stream)
+                marks.append(e)
+        mark()
+        mover.pack(buckets, cks_fused)
+        mark()
+        mover.checksum(buckets, cks_alone)
+        mark()
+        unmover.unpack(buckets)
+        mark()
+        for ex, out in shards:
+            ex.extract(out)
+        mark()
+        if events is not None:
+            events.append(marks)
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = binding.tm_launch_count()
+    op_events: List[list] = []
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record(stream)
+    for _ in range(args.steps):
+        one_step(op_events)
+    end.record(stream)
+    torch.cuda.synchronize()
+    elapsed_ms = start.elapsed_time(end)
+    launches = binding.tm_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        dist.barrier()
+        torch.cuda.synchronize()
+    assert mover.status() == 0 and unmover.status() == 0
+    ok = bool(torch.equal(cks_fused, cks_alone))
+    ok = ok and all(torch.equal(a, b) for a, b in zip(state.tensors[:8], target.tensors[:8]))
+
+    total_ms, total_bytes = aggregate_over_ranks(elapsed_ms, bytes_per_step * args.steps)
+
+    names = ["pack", "checksum", "unpack", "shard"]
+    op_ms = {n: statistics.mean(m[i].elapsed_time(m[i + 1]) for m in op_events) for i, n in enumerate(names)}
+    peak, peak_kind = measured_hbm_peak()
+    ops = {n: {"ms": round(op_ms[n], 4), "GB/s": round(gbs(per_op[n], op_ms[n]), 1),
+               "frac_of_measured_copy": round(gbs(per_op[n], op_ms[n]) / peak, 4),
+               "frac_of_8TBs_nominal": round(gbs(per_op[n], op_ms[n]) / NOMINAL_HBM_GBS, 4)} for n in names}
+    pcs_bytes = per_op["pack"] + per_op["shard"]
+    pcs_ms = op_ms["pack"] + op_ms["shard"]
+    ops["pack+checksum+shard"] = {"ms": round(pcs_ms, 4), "GB/s": round(gbs(pcs_bytes, pcs_ms), 1),
+                                  "frac_of_measured_copy": round(gbs(pcs_bytes, pcs_ms) / peak, 4),
+                                  "frac_of_8TBs_nominal": round(gbs(pcs_bytes, pcs_ms) / NOMINAL_HBM_GBS, 4)}
+    achieved = gbs(per_op["pack"], op_ms["pack"])
+    roofline = {"bound": "hbm", "kernel": "pack_kernel (fused pack + checksum)", "achieved": round(achieved, 1),
+                "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "traffic": None, "algorithmic_bytes_per_launch": per_op["pack"]}
+
+    e2e = None
+    cpu_baseline = None
+    if rank == 0 and world == 1:
+        e2e = run_e2e(args, cfg, state, mover, buckets, cks_fused, bytes_per_step, one_step, shards)
+        if not args.no_cpu_baseline:
+            step, sample = oracle_sample_step(cfg)
+            dt, nb = step()
+            cpu_baseline = {"value": round(gbs(nb, dt * 1e3), 4), "unit": UNIT, "cores": 1, "kind": "oracle",
+                            "sample": sample, "seconds": round(dt, 2), "host_cores_available": os.cpu_count()}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    line = {
+        "metric": METRIC, "value": round(gbs(total_bytes, total_ms), 2), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8/u64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}:{cfg.name}", "state_bytes": state.state_bytes,
+                   "bucket_bytes": cfg.bucket_bytes, "n_buckets": mover.n_buckets, "n_tensors": len(state.specs),
+                   "shard": f"r={cfg.shard_r} of D={cfg.shard_D}, three fp32 planes", "parallelism": "replicas only",
+                   "l2": "inputs (GBs) far larger than the 126 MB L2; no flush needed",
+                   "step": "pack+fused checksum, stand-alone checksum, unpack, shard extract x3"},
+        "bytes_per_step": bytes_per_step, "ops": ops, "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "self_check": "ok" if ok else "MISMATCH",
+        "frac_of_8TBs_nominal": round(gbs(total_bytes, total_ms) / NOMINAL_HBM_GBS / world, 4),
+    }
+    print(json.dumps(line), flush=True)
+    if not ok:
+        raise SystemExit("self-check failed: fused and stand-alone checksums differ or round trip broke")
+
+
+def run_e2e(args, cfg, state, mover, buckets, cks, bytes_per_step, one_step, shards):
+    """Same step, but the role's tensors start in pinned host memory and the results (packed stream,
+    checksums, shards) end in pinned host memory; the copies are inside the timed region."""
+    try:
+        import psutil
+        avail = psutil.virtual_memory().available
+    except Exception:
+        avail = 0
+    h2d = state.state_bytes
+    d2h = mover.total_bytes + 8 * mover.n_buckets + sum(ex.out_bytes for ex, _ in shards)
+    if avail < 2 * (h2d + d2h) + (8 << 30):
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "skipped": f"host has {avail >> 30} GiB available, pinned staging needs {(h2d + d2h) >> 30} GiB"}
+    from paper_2412_12636_b200 import layouts
+    host_in = torch.empty(h2d, dtype=torch.uint8, pin_memory=True)
+    host_out = torch.empty(d2h, dtype=torch.uint8, pin_memory=True)
+    views, pos = [], 0
+    for t in state.tensors:
+        n = t.numel() * t.element_size()
+        v = host_in[pos:pos + n]
+        v.copy_(layouts.tensor_bytes(t))
+        views.append(v)
+        pos += n
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    def e2e_step():
+        for t, v in zip(state.tensors, views):
+            layouts.tensor_bytes(t).copy_(v, non_blocking=True)
+        one_step()
+        o = 0
+        host_out[o:o + mover.total_bytes].copy_(buckets, non_blocking=True)
+        o += mover.total_bytes
+        host_out[o:o + 8 * mover.n_buckets].copy_(cks.view(torch.uint8), non_blocking=True)
+        o += 8 * mover.n_buckets
+        for ex, out in shards:
+            host_out[o:o + ex.out_bytes].copy_(out, non_blocking=True)
+            o += ex.out_bytes
+
+    e2e_step()
+    torch.cuda.synchronize()
+    k = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record(stream)
+    for _ in range(k):
+        e2e_step()
+    e.record(stream)
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - t0) * 1e3 / k
+    ms = s.elapsed_time(e) / k
+    return {"value": round(gbs(bytes_per_step, max(ms, wall_ms)), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": round(max(ms, wall_ms), 3), "steps": k,
+            "note": "role tensors start and results end in pinned host memory; PCIe-bound"}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg3")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

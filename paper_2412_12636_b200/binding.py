@@ -1,0 +1,174 @@
+"""Thin ctypes binding of the C-ABI library (include/tm_state.h): argument marshalling only.
+
+Every function takes raw device addresses (ints, e.g. ``tensor.data_ptr()``) and a raw stream
+handle (``torch.cuda.current_stream().cuda_stream``); every step of the path runs in the library's
+kernels.  There is no CPU fallback: if ``libtm_state.so`` has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Iterable, List, Optional, Sequence, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtm_state.so")
+
+TM_OK = 0
+TM_ERR_ARG, TM_ERR_ALIGN, TM_ERR_CAPACITY, TM_ERR_OVERLAP = -1, -2, -3, -4
+TM_ERR_RANK, TM_ERR_DTYPE, TM_ERR_CUDA, TM_ERR_TIMEOUT, TM_ERR_STATE = -5, -6, -7, -8, -9
+
+_u64, _u32, _p, _int = ctypes.c_uint64, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_int
+
+# every symbol include/tm_state.h declares: name -> (restype, argtypes)
+SIGNATURES = {
+    "tm_plan_create": (_int, [_p, _u64, _u64, _p]),
+    "tm_plan_query": (_int, [_p, _p, _p, _p]),
+    "tm_plan_offsets": (_int, [_p, _p]),
+    "tm_plan_upload": (_int, [_p, _p, _u64, _p]),
+    "tm_plan_status": (_int, [_p, _p, _p]),
+    "tm_plan_destroy": (None, [_p]),
+    "tm_state_pack": (_int, [_p, _p, _u64, _p, _p]),
+    "tm_state_unpack": (_int, [_p, _p, _u64, _p]),
+    "tm_shard_bounds": (_int, [_u64, _u32, _u32, _p, _p]),
+    "tm_shard_workspace": (_int, [_p, _u64, _u32, _u32, _p]),
+    "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
+    "tm_workspace_status": (_int, [_p, _p, _p]),
+    "tm_checksum": (_int, [_p, _u64, _u64, _p, _p]),
+    "tm_strerror": (ctypes.c_char_p, [_int]),
+    "tm_last_cuda_error": (_int, []),
+    "tm_launch_count": (_u64, []),
+}
+
+
+class TmDesc(ctypes.Structure):
+    _fields_ = [("ptr", _p), ("nbytes", _u64), ("elem_size", _u32), ("plane", _u32)]
+
+
+class TmError(RuntimeError):
+    def __init__(self, status: int, what: str, detail: str = ""):
+        super().__init__(f"{what}: {detail or status} (status {status})")
+        self.status = status
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libtm_state.so; raises if it is missing (build it with paper_2412_12636_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: the CUDA library has not been built "
+                              "(run `python paper_2412_12636_b200/build.py`); there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, what: str) -> None:
+    if status != TM_OK:
+        L = load_library()
+        detail = L.tm_strerror(status).decode()
+        if status == TM_ERR_CUDA:
+            detail += f" (cudaError {L.tm_last_cuda_error()})"
+        raise TmError(status, what, detail)
+
+
+def make_descs(descs: Iterable[Tuple[int, int, int, int]]):
+    """ctypes array of tm_desc from (address, nbytes, elem_size, plane) tuples."""
+    descs = list(descs)
+    arr = (TmDesc * len(descs))()
+    for i, (ptr, nbytes, elem_size, plane) in enumerate(descs):
+        arr[i].ptr, arr[i].nbytes, arr[i].elem_size, arr[i].plane = ptr, nbytes, elem_size, plane
+    return arr
+
+
+class Plan:
+    """Owner of a tm_plan handle."""
+
+    def __init__(self, descs: Sequence[Tuple[int, int, int, int]], bucket_bytes: int):
+        L = load_library()
+        self._h = _p()
+        arr = make_descs(descs)
+        _check(L.tm_plan_create(arr, len(arr), bucket_bytes, ctypes.byref(self._h)), "tm_plan_create")
+        self.n_desc = len(arr)
+        t, n, w = _u64(), _u64(), _u64()
+        _check(L.tm_plan_query(self._h, ctypes.byref(t), ctypes.byref(n), ctypes.byref(w)), "tm_plan_query")
+        self.total_bytes, self.n_buckets, self.workspace_bytes = t.value, n.value, w.value
+        self.bucket_bytes = bucket_bytes
+
+    def offsets(self) -> List[int]:
+        out = (_u64 * self.n_desc)()
+        _check(load_library().tm_plan_offsets(self._h, out), "tm_plan_offsets")
+        return list(out)
+
+    def upload(self, d_workspace: int, workspace_bytes: int, stream: int) -> None:
+        _check(load_library().tm_plan_upload(self._h, d_workspace, workspace_bytes, stream), "tm_plan_upload")
+
+    def status(self, stream: int) -> int:
+        s = _int()
+        _check(load_library().tm_plan_status(self._h, stream, ctypes.byref(s)), "tm_plan_status")
+        return s.value
+
+    @property
+    def handle(self):
+        return self._h
+
+    def close(self) -> None:
+        if self._h:
+            load_library().tm_plan_destroy(self._h)
+            self._h = _p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def tm_state_pack(plan: Plan, d_buckets: int, capacity: int, d_checksums: Optional[int], stream: int) -> None:
+    _check(load_library().tm_state_pack(plan.handle, d_buckets, capacity, d_checksums, stream), "tm_state_pack")
+
+
+def tm_state_unpack(plan: Plan, d_buckets: int, nbytes: int, stream: int) -> None:
+    _check(load_library().tm_state_unpack(plan.handle, d_buckets, nbytes, stream), "tm_state_unpack")
+
+
+def tm_shard_bounds(n_elems: int, r: int, D: int) -> Tuple[int, int]:
+    lo, hi = _u64(), _u64()
+    _check(load_library().tm_shard_bounds(n_elems, r, D, ctypes.byref(lo), ctypes.byref(hi)), "tm_shard_bounds")
+    return lo.value, hi.value
+
+
+def tm_shard_workspace(descs, r: int, D: int) -> int:
+    arr = descs if isinstance(descs, ctypes.Array) else make_descs(descs)
+    w = _u64()
+    _check(load_library().tm_shard_workspace(arr, len(arr), r, D, ctypes.byref(w)), "tm_shard_workspace")
+    return w.value
+
+
+def tm_shard_extract(descs, r: int, D: int, d_out: int, out_capacity: int, d_workspace: int,
+                     workspace_bytes: int, stream: int) -> int:
+    """Returns the number of elements written."""
+    arr = descs if isinstance(descs, ctypes.Array) else make_descs(descs)
+    n = _u64()
+    _check(load_library().tm_shard_extract(arr, len(arr), r, D, d_out, out_capacity, ctypes.byref(n),
+                                           d_workspace, workspace_bytes, stream), "tm_shard_extract")
+    return n.value
+
+
+def tm_workspace_status(d_workspace: int, stream: int) -> int:
+    s = _int()
+    _check(load_library().tm_workspace_status(d_workspace, stream, ctypes.byref(s)), "tm_workspace_status")
+    return s.value
+
+
+def tm_checksum(d_bytes: int, nbytes: int, bucket_bytes: int, d_checksums: int, stream: int) -> None:
+    _check(load_library().tm_checksum(d_bytes, nbytes, bucket_bytes, d_checksums, stream), "tm_checksum")
+
+
+def tm_launch_count() -> int:
+    return load_library().tm_launch_count()

@@ -1,0 +1,238 @@
+// C ABI of the role-state mover (declared in include/tm_state.h): argument validation, work-list
+// upload and kernel launches.  Nothing here computes on the CPU what the kernels are for; without
+// a CUDA device every operation fails with TM_ERR_CUDA.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstring>
+#include <new>
+
+#include "tm_internal.h"
+
+int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes);
+int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
+int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                      uint32_t* elem_size, uint64_t* n_elems);
+void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
+                       uint64_t d_out, tms::WorkList* wl);
+int tm_targets_disjoint(const tm_plan* p);
+
+namespace {
+
+std::atomic<int> g_last_cuda_error{0};
+
+int cuda_fail(int e) {
+  g_last_cuda_error.store(e);
+  return TM_ERR_CUDA;
+}
+#define TM_CUDA(call)                              \
+  do {                                             \
+    cudaError_t e__ = (call);                      \
+    if (e__ != cudaSuccess) return cuda_fail((int)e__); \
+  } while (0)
+
+bool ranges_overlap(uint64_t a, uint64_t an, uint64_t b, uint64_t bn) {
+  return a < b + bn && b < a + an;
+}
+
+int upload_worklist(const tms::WorkList& wl, const tms::WorkspaceLayout& l, uint8_t* d_ws, cudaStream_t st) {
+  TM_CUDA(cudaMemsetAsync(d_ws, 0, tms::kStatusBlockBytes, st));
+  if (!wl.segs.empty())
+    TM_CUDA(cudaMemcpyAsync(d_ws + l.segs_off, wl.segs.data(), wl.segs.size() * sizeof(tms::Seg),
+                            cudaMemcpyHostToDevice, st));
+  TM_CUDA(cudaMemcpyAsync(d_ws + l.items_off, wl.item_first.data(),
+                          wl.item_first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+  return TM_OK;
+}
+
+int read_status(const void* d_ws, cudaStream_t st, int* device_status) {
+  if (d_ws == nullptr || device_status == nullptr) return TM_ERR_ARG;
+  int word = 0;
+  TM_CUDA(cudaMemcpyAsync(&word, d_ws, sizeof(int), cudaMemcpyDeviceToHost, st));
+  TM_CUDA(cudaStreamSynchronize(st));
+  *device_status = word;
+  return TM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int tm_plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_plan** out) {
+  if (out == nullptr) return TM_ERR_ARG;
+  *out = nullptr;
+  tm_plan* p = new (std::nothrow) tm_plan();
+  if (p == nullptr) return TM_ERR_ARG;
+  int rc = tm_plan_build(p, descs, n_desc, bucket_bytes);
+  if (rc != TM_OK) {
+    delete p;
+    return rc;
+  }
+  *out = p;
+  return TM_OK;
+}
+
+int tm_plan_query(const tm_plan* plan, uint64_t* total_bytes, uint64_t* n_buckets,
+                  uint64_t* workspace_bytes) {
+  if (plan == nullptr) return TM_ERR_ARG;
+  if (total_bytes != nullptr) *total_bytes = plan->total_bytes;
+  if (n_buckets != nullptr) *n_buckets = plan->n_buckets;
+  if (workspace_bytes != nullptr) *workspace_bytes = plan->ws_layout.total;
+  return TM_OK;
+}
+
+int tm_plan_offsets(const tm_plan* plan, uint64_t* offsets) {
+  if (plan == nullptr || offsets == nullptr) return TM_ERR_ARG;
+  std::memcpy(offsets, plan->offsets.data(), plan->offsets.size() * sizeof(uint64_t));
+  return TM_OK;
+}
+
+int tm_plan_upload(tm_plan* plan, void* d_workspace, uint64_t workspace_bytes, void* stream) {
+  if (plan == nullptr || d_workspace == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+  if (workspace_bytes < plan->ws_layout.total) return TM_ERR_CAPACITY;
+  int rc = upload_worklist(plan->work, plan->ws_layout, (uint8_t*)d_workspace, (cudaStream_t)stream);
+  if (rc != TM_OK) return rc;
+  plan->d_workspace = (uint8_t*)d_workspace;
+  return TM_OK;
+}
+
+int tm_plan_status(const tm_plan* plan, void* stream, int* device_status) {
+  if (plan == nullptr) return TM_ERR_ARG;
+  if (plan->d_workspace == nullptr) return TM_ERR_STATE;
+  return read_status(plan->d_workspace, (cudaStream_t)stream, device_status);
+}
+
+void tm_plan_destroy(tm_plan* plan) { delete plan; }
+
+int tm_state_pack(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint64_t* d_checksums,
+                  void* stream) {
+  if (plan == nullptr || d_buckets == nullptr) return TM_ERR_ARG;
+  if (plan->d_workspace == nullptr) return TM_ERR_STATE;
+  if (((uintptr_t)d_buckets & 255) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
+  if (capacity < plan->total_bytes) return TM_ERR_CAPACITY;
+  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
+  for (const tm_desc& d : plan->descs)
+    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (d_checksums != nullptr)
+    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), st));
+  const uint8_t* ws = plan->d_workspace;
+  int e = tms::launch_pack((const tms::Seg*)(ws + plan->ws_layout.segs_off),
+                          (const uint32_t*)(ws + plan->ws_layout.items_off),
+                          (uint32_t)plan->work.n_items(), (uint8_t*)d_buckets,
+                          (unsigned long long*)d_checksums, (int*)plan->d_workspace, stream);
+  return e == 0 ? TM_OK : cuda_fail(e);
+}
+
+int tm_state_unpack(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, void* stream) {
+  if (plan == nullptr || d_buckets == nullptr) return TM_ERR_ARG;
+  if (plan->d_workspace == nullptr) return TM_ERR_STATE;
+  if (((uintptr_t)d_buckets & 255) != 0) return TM_ERR_ALIGN;
+  if (nbytes < plan->total_bytes) return TM_ERR_CAPACITY;
+  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
+  for (const tm_desc& d : plan->descs)
+    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
+  if (plan->targets_disjoint == 0) plan->targets_disjoint = tm_targets_disjoint(plan);
+  if (plan->targets_disjoint < 0) return TM_ERR_OVERLAP;
+  const uint8_t* ws = plan->d_workspace;
+  int e = tms::launch_copy((const tms::Seg*)(ws + plan->ws_layout.segs_off),
+                          (const uint32_t*)(ws + plan->ws_layout.items_off),
+                          (uint32_t)plan->work.n_items(), (uint8_t*)const_cast<void*>(d_buckets),
+                          /*to_tensors=*/true, (int*)plan->d_workspace, stream);
+  return e == 0 ? TM_OK : cuda_fail(e);
+}
+
+int tm_shard_bounds(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi) {
+  if (lo == nullptr || hi == nullptr) return TM_ERR_ARG;
+  return tm_bounds_u128(n_elems, r, D, lo, hi);
+}
+
+int tm_shard_workspace(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                       uint64_t* workspace_bytes) {
+  if (workspace_bytes == nullptr) return TM_ERR_ARG;
+  uint32_t e = 0;
+  uint64_t n_elems = 0;
+  int rc = tm_shard_validate(plane_descs, n_desc, r, D, &e, &n_elems);
+  if (rc != TM_OK) return rc;
+  uint64_t lo = 0, hi = 0;
+  rc = tm_bounds_u128(n_elems, r, D, &lo, &hi);
+  if (rc != TM_OK) return rc;
+  // upper bound on pieces: every tensor adds at most two partial pieces to the chunk count
+  const uint64_t chunk = tms::tuning().chunk_bytes;
+  const uint64_t max_segs = (hi - lo) * e / chunk + 2 * n_desc + 2;
+  *workspace_bytes = tms::workspace_layout(max_segs, max_segs).total;
+  return TM_OK;
+}
+
+int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, void* d_out,
+                     uint64_t out_capacity, uint64_t* out_elems, void* d_workspace,
+                     uint64_t workspace_bytes, void* stream) {
+  uint32_t e = 0;
+  uint64_t n_elems = 0;
+  int rc = tm_shard_validate(plane_descs, n_desc, r, D, &e, &n_elems);
+  if (rc != TM_OK) return rc;
+  uint64_t lo = 0, hi = 0;
+  rc = tm_bounds_u128(n_elems, r, D, &lo, &hi);
+  if (rc != TM_OK) return rc;
+  if (out_elems != nullptr) *out_elems = hi - lo;
+  if (hi == lo) return TM_OK;
+  if (d_out == nullptr || d_workspace == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_out & 1) != 0 || ((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+  const uint64_t out_bytes = (hi - lo) * e;
+  if (out_capacity < out_bytes) return TM_ERR_CAPACITY;
+  const uint64_t out_addr = (uint64_t)(uintptr_t)d_out;
+  for (uint64_t k = 0; k < n_desc; ++k)
+    if (ranges_overlap((uint64_t)(uintptr_t)plane_descs[k].ptr, plane_descs[k].nbytes, out_addr, out_bytes))
+      return TM_ERR_OVERLAP;
+  tms::WorkList wl;
+  tm_shard_worklist(plane_descs, n_desc, e, lo, hi, out_addr, &wl);
+  const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
+  if (workspace_bytes < l.total) return TM_ERR_CAPACITY;
+  rc = upload_worklist(wl, l, (uint8_t*)d_workspace, (cudaStream_t)stream);
+  if (rc != TM_OK) return rc;
+  const uint8_t* ws = (const uint8_t*)d_workspace;
+  int err = tms::launch_copy((const tms::Seg*)(ws + l.segs_off), (const uint32_t*)(ws + l.items_off),
+                            (uint32_t)wl.n_items(), (uint8_t*)d_out, /*to_tensors=*/false,
+                            (int*)d_workspace, stream);
+  return err == 0 ? TM_OK : cuda_fail(err);
+}
+
+int tm_workspace_status(const void* d_workspace, void* stream, int* device_status) {
+  return read_status(d_workspace, (cudaStream_t)stream, device_status);
+}
+
+int tm_checksum(const void* d_bytes, uint64_t nbytes, uint64_t bucket_bytes, uint64_t* d_checksums,
+                void* stream) {
+  if (bucket_bytes == 0 || bucket_bytes > (1ull << 35)) return TM_ERR_ARG;
+  if (bucket_bytes % 256 != 0) return TM_ERR_ALIGN;
+  if (nbytes == 0) return TM_OK;
+  if (d_bytes == nullptr || d_checksums == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_bytes & 15) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
+  const uint64_t n_buckets = (nbytes + bucket_bytes - 1) / bucket_bytes;
+  cudaStream_t st = (cudaStream_t)stream;
+  TM_CUDA(cudaMemsetAsync(d_checksums, 0, n_buckets * sizeof(uint64_t), st));
+  int e = tms::launch_checksum((const uint8_t*)d_bytes, nbytes, bucket_bytes,
+                              (unsigned long long*)d_checksums, stream);
+  return e == 0 ? TM_OK : cuda_fail(e);
+}
+
+const char* tm_strerror(int status) {
+  switch (status) {
+    case TM_OK: return "ok";
+    case TM_ERR_ARG: return "invalid argument";
+    case TM_ERR_ALIGN: return "misaligned address or bucket size";
+    case TM_ERR_CAPACITY: return "buffer too small";
+    case TM_ERR_OVERLAP: return "buffers overlap";
+    case TM_ERR_RANK: return "invalid shard rank";
+    case TM_ERR_DTYPE: return "unsupported or mixed element size";
+    case TM_ERR_CUDA: return "CUDA runtime error";
+    case TM_ERR_TIMEOUT: return "bounded device wait expired";
+    case TM_ERR_STATE: return "plan has no uploaded work list";
+    default: return "unknown status";
+  }
+}
+
+int tm_last_cuda_error(void) { return g_last_cuda_error.load(); }
+
+}  // extern "C"

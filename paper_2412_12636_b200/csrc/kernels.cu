@@ -1,0 +1,363 @@
+// sm_100a kernels of the role-state mover: fused pack + checksum, generic piece copy (unpack and
+// shard extract) and stand-alone checksum.  Everything here is HBM-bound byte movement with one
+// 64-bit multiply-add per 8 bytes; there is no contraction, so no tensor cores.
+//
+// Work distribution: a persistent grid walks the item list with a grid stride.  An item with one
+// piece is copied by the whole block; an item with several small pieces gives one warp per piece.
+// All global accesses of the main loops are 16-byte vectors, consecutive lanes on consecutive
+// vectors.  A piece whose tensor address is not 16-byte aligned is read as aligned vectors and
+// re-aligned in registers (funnel shifts), so stores and checksum words stay aligned to the flat
+// buffer.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "tm_internal.h"
+
+namespace tms {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kUnroll = 4;         // independent 16-byte loads in flight per thread, aligned sources
+constexpr int kUnrollShifted = 2;  // same for sources that need re-alignment (two loads per vector)
+constexpr int kMinBlocks = 4;  // resident blocks per SM the register budget is held to
+
+typedef unsigned long long u64;
+
+// ---- streaming 16-byte accesses -----------------------------------------------------------------
+// Data is touched once: loads bypass L1 allocation, stores are marked streaming.
+__device__ __forceinline__ uint4 ld16(const uint8_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+// Lines that neighbouring threads read twice (misaligned sources) may stay in L1.
+__device__ __forceinline__ uint4 ld16_cached(const uint8_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st16(uint8_t* p, uint4 v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+               "r"(v.w)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t ld2(const uint8_t* p) {
+  return (uint32_t)(*reinterpret_cast<const uint16_t*>(p));
+}
+__device__ __forceinline__ void st2(uint8_t* p, uint32_t v) {
+  *reinterpret_cast<uint16_t*>(p) = (uint16_t)v;
+}
+
+// Vector v of a source that starts `a` bytes (even, 2..14) after the aligned address `sa`: bytes
+// [16v + a, 16v + a + 16) of the aligned stream, taken from two aligned vectors with a barrel
+// shifter: whole words by ws = a / 4 (two select stages), then bits by bs = 8 * (a mod 4).
+__device__ __forceinline__ uint4 ld16_shifted(const uint8_t* sa, uint32_t v, uint32_t ws, uint32_t bs) {
+  const uint4 lo = ld16_cached(sa + (size_t)v * 16);
+  const uint4 hi = ld16_cached(sa + (size_t)v * 16 + 16);
+  uint32_t c0 = lo.x, c1 = lo.y, c2 = lo.z, c3 = lo.w, c4 = hi.x, c5 = hi.y, c6 = hi.z, c7 = hi.w;
+  if (ws & 2) { c0 = c2; c1 = c3; c2 = c4; c3 = c5; c4 = c6; c5 = c7; }
+  if (ws & 1) { c0 = c1; c1 = c2; c2 = c3; c3 = c4; c4 = c5; }
+  uint4 r;
+  r.x = __funnelshift_r(c0, c1, bs);
+  r.y = __funnelshift_r(c1, c2, bs);
+  r.z = __funnelshift_r(c2, c3, bs);
+  r.w = __funnelshift_r(c3, c4, bs);
+  return r;
+}
+
+// Running checksum state of one thread.  Within a piece the weight of local word j is 2j+1
+// (fits 32 bits: pieces are < 4 GiB); the piece's position in its bucket enters once at the end:
+//   sum_j w_j * (2*(word0 + j) + 1) = sum_j w_j * (2j+1) + 2*word0 * sum_j w_j.
+struct Cksum {
+  u64 acc = 0;  // sum of w_j * (2j+1)
+  u64 sw = 0;   // sum of w_j
+  __device__ __forceinline__ void add(uint4 x, uint32_t v) {
+    const u64 w0 = (u64)x.x | ((u64)x.y << 32);
+    const u64 w1 = (u64)x.z | ((u64)x.w << 32);
+    const uint32_t k = 4u * v + 1u;  // weight of local word 2v; word 2v+1 has k + 2
+    acc += w0 * (u64)k + w1 * (u64)(k + 2u);
+    sw += w0 + w1;
+  }
+  __device__ __forceinline__ u64 finish(uint32_t word0) {
+    const u64 r = acc + 2ull * (u64)word0 * sw;
+    acc = 0;
+    sw = 0;
+    return r;
+  }
+};
+
+// Copies full vectors [0, nfull) from src (any even alignment) to dst (16-byte aligned) with
+// threads g, g+G, ...; optionally accumulates the checksum of what is stored.
+template <bool CKSUM, bool ALIGNED>
+__device__ __forceinline__ void copy_vectors(uint8_t* dst, const uint8_t* src, uint32_t nfull, uint32_t g,
+                                             uint32_t G, uint32_t ws, uint32_t bs, Cksum& ck) {
+  constexpr int U = ALIGNED ? kUnroll : kUnrollShifted;
+  const uint8_t* sa = src - (ALIGNED ? 0 : ((uintptr_t)src & 15));
+  for (uint32_t v0 = g; v0 < nfull; v0 += G * U) {
+    uint4 x[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t v = v0 + u * G;
+      if (v < nfull) x[u] = ALIGNED ? ld16(sa + (size_t)v * 16) : ld16_shifted(sa, v, ws, bs);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t v = v0 + u * G;
+      if (v < nfull) {
+        st16(dst + (size_t)v * 16, x[u]);
+        if (CKSUM) ck.add(x[u], v);
+      }
+    }
+  }
+}
+
+template <bool CKSUM>
+__device__ __forceinline__ void copy_vectors_any(uint8_t* dst, const uint8_t* src, uint32_t nfull,
+                                                 uint32_t g, uint32_t G, Cksum& ck) {
+  const uint32_t a = (uint32_t)((uintptr_t)src & 15);   // uniform over the group
+  if (a == 0) copy_vectors<CKSUM, true>(dst, src, nfull, g, G, 0, 0, ck);
+  else copy_vectors<CKSUM, false>(dst, src, nfull, g, G, a >> 2, (a & 3) * 8, ck);
+}
+
+// Pack one piece: tensor -> stream, zero padding, checksum.  dst is 256-byte aligned.
+__device__ __forceinline__ void pack_piece(const Seg& s, uint8_t* stream, uint32_t g, uint32_t G, Cksum& ck) {
+  uint8_t* dst = stream + s.off;
+  const uint8_t* src = reinterpret_cast<const uint8_t*>(s.tensor);
+  const uint32_t n = s.nbytes;
+  const uint32_t nfull = n >> 4;
+  copy_vectors_any<true>(dst, src, nfull, g, G, ck);
+  // the vector that holds the tensor's last (n mod 16) bytes, then whole vectors of padding
+  const uint32_t nvec = (n + s.pad) >> 4;
+  const uint32_t rem = n & 15;
+  for (uint32_t v = nfull + g; v < nvec; v += G) {
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    if (v == nfull && rem != 0) {
+      const uint8_t* t = src + (size_t)nfull * 16;
+#pragma unroll
+      for (uint32_t h = 0; h < 7; ++h)
+        if (2 * h < rem) w[h >> 1] |= ld2(t + 2 * h) << ((h & 1) * 16);
+    }
+    const uint4 x = make_uint4(w[0], w[1], w[2], w[3]);
+    st16(dst + (size_t)v * 16, x);
+    ck.add(x, v);
+  }
+}
+
+// Copy one piece between a tensor and the flat buffer, both at any even alignment.
+__device__ __forceinline__ void copy_piece(uint8_t* dst, const uint8_t* src, uint32_t n, uint32_t g, uint32_t G) {
+  Cksum unused;
+  uint32_t head = (uint32_t)((0 - (uintptr_t)dst) & 15);
+  if (head > n) head = n;
+  if (2 * g < head) st2(dst + 2 * g, ld2(src + 2 * g));
+  dst += head;
+  src += head;
+  n -= head;
+  const uint32_t nfull = n >> 4;
+  copy_vectors_any<false>(dst, src, nfull, g, G, unused);
+  const uint32_t rem = n & 15;
+  const size_t t = (size_t)nfull * 16;
+  // the last G/… threads are as good as any; use the group's tail so the head threads differ
+  const uint32_t gt = G - 1 - g;
+  if (2 * gt < rem) st2(dst + t + 2 * gt, ld2(src + t + 2 * gt));
+}
+
+// Block-wide sum of a per-thread value, added to *target by one thread.
+__device__ __forceinline__ void block_flush(u64 value, u64* target, u64* smem) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) value += __shfl_xor_sync(0xffffffffu, value, o);
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) smem[warp] = value;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u64 total = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) total += smem[w];
+    if (total != 0) atomicAdd(target, total);
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads, kMinBlocks)
+pack_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
+            uint8_t* __restrict__ stream, u64* __restrict__ checksums) {
+  __shared__ u64 red[kWarps];
+  Cksum ck;
+  u64 total = 0;            // this thread's share of the checksum of bucket `cur`
+  uint32_t cur = 0xffffffffu;
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t first = item_first[item], last = item_first[item + 1];
+    const uint32_t bucket = segs[first].bucket;
+    if (bucket != cur) {    // uniform over the block
+      if (cur != 0xffffffffu && checksums != nullptr) block_flush(total, checksums + cur, red);
+      total = 0;
+      cur = bucket;
+    }
+    // one piece: the whole block copies it; several pieces: one warp per piece
+    const bool single = (last - first == 1);
+    const uint32_t g = single ? threadIdx.x : lane, G = single ? kThreads : 32u;
+    for (uint32_t i = first + (single ? 0u : warp); i < last; i += (single ? 1u : (uint32_t)kWarps)) {
+      const Seg s = segs[i];
+      pack_piece(s, stream, g, G, ck);
+      total += ck.finish(s.word0);
+    }
+  }
+  if (cur != 0xffffffffu && checksums != nullptr) block_flush(total, checksums + cur, red);
+}
+
+template <bool TO_TENSORS>
+__global__ void __launch_bounds__(kThreads, kMinBlocks)
+copy_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
+            uint8_t* __restrict__ flat) {
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t first = item_first[item], last = item_first[item + 1];
+    const bool single = (last - first == 1);
+    const uint32_t g = single ? threadIdx.x : lane, G = single ? kThreads : 32u;
+    for (uint32_t i = first + (single ? 0u : warp); i < last; i += (single ? 1u : (uint32_t)kWarps)) {
+      const Seg s = segs[i];
+      uint8_t* t = reinterpret_cast<uint8_t*>(s.tensor);
+      uint8_t* f = flat + s.off;
+      copy_piece(TO_TENSORS ? t : f, TO_TENSORS ? f : t, s.nbytes, g, G);
+    }
+  }
+}
+
+// Stand-alone checksum.  Tile t covers bytes [tile_bytes * (t % tiles_per_bucket), +tile_bytes) of
+// bucket t / tiles_per_bucket.  The input is 16-byte aligned; only the very last vector of the
+// input can be partial.
+constexpr uint32_t kCksumTile = 64 * 1024;
+
+__global__ void __launch_bounds__(kThreads, kMinBlocks)
+checksum_kernel(const uint8_t* __restrict__ bytes, u64 nbytes, u64 bucket_bytes, uint32_t tiles_per_bucket,
+                u64 n_tiles, u64* __restrict__ checksums) {
+  __shared__ u64 red[kWarps];
+  Cksum ck;
+  u64 total = 0;
+  u64 cur = ~0ull;
+  for (u64 t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    const u64 bucket = t / tiles_per_bucket;
+    const u64 in_bucket = (t - bucket * tiles_per_bucket) * (u64)kCksumTile;
+    const u64 begin = bucket * bucket_bytes + in_bucket;
+    u64 end = begin + kCksumTile;
+    const u64 bucket_end = (bucket + 1) * bucket_bytes;
+    if (end > bucket_end) end = bucket_end;
+    if (end > nbytes) end = nbytes;
+    if (in_bucket >= bucket_bytes || begin >= end) continue;   // uniform over the block
+    if (bucket != cur) {
+      if (cur != ~0ull) block_flush(total, checksums + cur, red);
+      total = 0;
+      cur = bucket;
+    }
+    const uint8_t* p = bytes + begin;
+    const uint32_t n = (uint32_t)(end - begin);
+    const uint32_t nfull = n >> 4;
+    for (uint32_t v0 = threadIdx.x; v0 < nfull; v0 += kThreads * kUnroll) {
+      uint4 x[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const uint32_t v = v0 + u * kThreads;
+        if (v < nfull) x[u] = ld16(p + (size_t)v * 16);
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const uint32_t v = v0 + u * kThreads;
+        if (v < nfull) ck.add(x[u], v);
+      }
+    }
+    const uint32_t rem = n & 15;
+    if (rem != 0 && threadIdx.x == 0) {   // ragged end of the input: assemble the last bytes
+      u64 w0 = 0, w1 = 0;
+      const uint8_t* q = p + (size_t)nfull * 16;
+      for (uint32_t b = 0; b < rem; ++b) {
+        if (b < 8) w0 |= (u64)q[b] << (8 * b);
+        else w1 |= (u64)q[b] << (8 * (b - 8));
+      }
+      ck.add(make_uint4((uint32_t)w0, (uint32_t)(w0 >> 32), (uint32_t)w1, (uint32_t)(w1 >> 32)), nfull);
+    }
+    total += ck.finish((uint32_t)(in_bucket / 8));
+  }
+  if (cur != ~0ull) block_flush(total, checksums + cur, red);
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+uint64_t launches() { return g_launches.load(std::memory_order_relaxed); }
+
+int device_sm_count(int* sms) {
+  static int cached[64] = {0};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return (int)e;
+  if (dev >= 0 && dev < 64 && cached[dev] > 0) {
+    *sms = cached[dev];
+    return 0;
+  }
+  int n = 0;
+  e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return (int)e;
+  if (dev >= 0 && dev < 64) cached[dev] = n;
+  *sms = n;
+  return 0;
+}
+
+static int grid_for(uint64_t n_items, uint32_t* grid) {
+  int sms = 0;
+  int rc = device_sm_count(&sms);
+  if (rc != 0) return rc;
+  uint64_t g = (uint64_t)sms * tuning().ctas_per_sm;
+  if (g > n_items) g = n_items;
+  if (g == 0) g = 1;
+  *grid = (uint32_t)g;
+  return 0;
+}
+
+int launch_pack(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
+                unsigned long long* d_checksums, int* /*d_status*/, void* stream) {
+  uint32_t grid = 0;
+  int rc = grid_for(n_items, &grid);
+  if (rc != 0) return rc;
+  pack_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_stream,
+                                                          d_checksums);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_copy(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
+                bool to_tensors, int* /*d_status*/, void* stream) {
+  uint32_t grid = 0;
+  int rc = grid_for(n_items, &grid);
+  if (rc != 0) return rc;
+  if (to_tensors)
+    copy_kernel<true><<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat);
+  else
+    copy_kernel<false><<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_checksum(const uint8_t* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
+                    unsigned long long* d_checksums, void* stream) {
+  const uint64_t n_buckets = (nbytes + bucket_bytes - 1) / bucket_bytes;
+  const uint64_t tpb = (bucket_bytes + kCksumTile - 1) / kCksumTile;
+  const uint64_t n_tiles = n_buckets * tpb;
+  uint32_t grid = 0;
+  int rc = grid_for(n_tiles, &grid);
+  if (rc != 0) return rc;
+  checksum_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_bytes, nbytes, bucket_bytes, (uint32_t)tpb,
+                                                              n_tiles, d_checksums);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+}  // namespace tms
+
+extern "C" uint64_t tm_launch_count(void) { return tms::launches(); }

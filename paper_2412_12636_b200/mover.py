@@ -1,0 +1,74 @@
+"""Convenience owners of device buffers around the C-ABI calls.  PyTorch supplies device memory
+and streams only; all data movement and checksum arithmetic happens inside the library."""
+from __future__ import annotations
+
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+from . import binding
+
+
+def _stream_handle(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+class RoleMover:
+    """A packed-stream plan for one role's tensors with its uploaded work list."""
+
+    def __init__(self, descs: Sequence[Tuple[int, int, int, int]], bucket_bytes: int, device="cuda",
+                 stream: Optional[torch.cuda.Stream] = None):
+        self.device = torch.device(device)
+        self.plan = binding.Plan(descs, bucket_bytes)
+        self.total_bytes = self.plan.total_bytes
+        self.n_buckets = self.plan.n_buckets
+        self.bucket_bytes = bucket_bytes
+        self.workspace = torch.empty(self.plan.workspace_bytes, dtype=torch.uint8, device=self.device)
+        self.plan.upload(self.workspace.data_ptr(), self.workspace.numel(), _stream_handle(stream))
+
+    def alloc_buckets(self) -> torch.Tensor:
+        return torch.empty(self.total_bytes, dtype=torch.uint8, device=self.device)
+
+    def alloc_checksums(self) -> torch.Tensor:
+        # uint64 values carried in an int64 tensor (bit pattern)
+        return torch.empty(self.n_buckets, dtype=torch.int64, device=self.device)
+
+    def pack(self, buckets: torch.Tensor, checksums: Optional[torch.Tensor] = None,
+             stream: Optional[torch.cuda.Stream] = None) -> None:
+        binding.tm_state_pack(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
+                              None if checksums is None else checksums.data_ptr(), _stream_handle(stream))
+
+    def unpack(self, buckets: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+        binding.tm_state_unpack(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
+                                _stream_handle(stream))
+
+    def checksum(self, buckets: torch.Tensor, checksums: torch.Tensor,
+                 stream: Optional[torch.cuda.Stream] = None) -> None:
+        binding.tm_checksum(buckets.data_ptr(), self.total_bytes, self.bucket_bytes, checksums.data_ptr(),
+                            _stream_handle(stream))
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        return self.plan.status(_stream_handle(stream))
+
+
+class ShardExtractor:
+    """Shard r of D of one plane (tensors of one element size), with its scratch workspace."""
+
+    def __init__(self, plane_descs: Sequence[Tuple[int, int, int, int]], r: int, D: int, device="cuda"):
+        self.device = torch.device(device)
+        self.descs = binding.make_descs(plane_descs)
+        self.r, self.D = r, D
+        self.elem_size = plane_descs[0][2]
+        n_elems = sum(d[1] for d in plane_descs) // self.elem_size
+        self.lo, self.hi = binding.tm_shard_bounds(n_elems, r, D)
+        self.out_bytes = (self.hi - self.lo) * self.elem_size
+        ws = binding.tm_shard_workspace(self.descs, r, D)
+        self.workspace = torch.empty(ws, dtype=torch.uint8, device=self.device)
+
+    def alloc_out(self) -> torch.Tensor:
+        return torch.empty(self.out_bytes, dtype=torch.uint8, device=self.device)
+
+    def extract(self, out: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+        return binding.tm_shard_extract(self.descs, self.r, self.D, out.data_ptr(),
+                                        out.numel() * out.element_size(), self.workspace.data_ptr(),
+                                        self.workspace.numel(), _stream_handle(stream))

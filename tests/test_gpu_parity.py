@@ -1,0 +1,173 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, must equal the CPU oracle bit for
+bit — every packed byte, every padding byte, every checksum, every unpacked tensor byte and every
+shard byte.  Integer and byte work only, so the bar is exact equality (no tolerance)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_12636_b200 import binding, layouts
+from paper_2412_12636_b200.mover import RoleMover, ShardExtractor
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _cuda():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.load_library()   # fails loudly if the CUDA library is not built
+    torch.cuda.set_device(0)
+    yield
+
+
+# ------------------------------------------------------------------ tiny and awkward layouts
+
+
+@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("B", [256, 512, 768, 1024, 1 << 20])
+def test_odd_layouts_pack_checksum_unpack(oracle_mod, seed, B):
+    specs = layouts.odd_specs(seed, n_tensors=3 + seed)
+    state = layouts.materialize_adversarial(specs, "cuda", seed=seed)   # 2-byte-granular addresses
+    G.check_pack_against_oracle(oracle_mod, state, B)
+
+
+@pytest.mark.parametrize("numel", [1, 2, 7, 8, 9, 127, 128, 129, 4095, 4096, 4097, 32767, 32768, 32769, 65535, 65537,
+                                   3 * 32768 + 5])
+@pytest.mark.parametrize("misalign", [0, 2, 4, 6, 8, 10, 12, 14])
+def test_single_tensor_every_alignment(oracle_mod, numel, misalign):
+    # bf16 elements: sizes around the vector (16 B), small-piece (8 KiB) and chunk (64 KiB) cuts
+    arena = torch.randint(0, 256, (2 * numel + 64,), dtype=torch.uint8, device="cuda",
+                          generator=torch.Generator("cuda").manual_seed(numel * 16 + misalign))
+    t = arena[misalign:misalign + 2 * numel]
+    spec = layouts.TensorSpec("t", numel, torch.bfloat16, 0, 0)
+    state = layouts.RoleState("one", [spec], [t], 1 << 20, 0, 1, arena)
+    G.check_pack_against_oracle(oracle_mod, state, 4096)
+
+
+def test_tensor_straddles_many_buckets_and_exact_fit(oracle_mod):
+    gen = torch.Generator("cuda").manual_seed(5)
+    a = torch.randint(0, 256, (10 * 4096,), dtype=torch.uint8, device="cuda", generator=gen)   # exactly 10 buckets
+    b = torch.randint(0, 256, (4096 + 2,), dtype=torch.uint8, device="cuda", generator=gen)
+    specs = [layouts.TensorSpec("a", a.numel() // 2, torch.bfloat16, 0, 0),
+             layouts.TensorSpec("b", b.numel() // 2, torch.bfloat16, 0, 1)]
+    state = layouts.RoleState("straddle", specs, [a, b], 4096, 0, 1)
+    mover, _, stream = G.check_pack_against_oracle(oracle_mod, state, 4096)
+    assert mover.n_buckets == 12 and stream.size == 11 * 4096 + 256
+    one = layouts.RoleState("fit", specs[:1], [a], 4096, 0, 1)
+    mover, _, stream = G.check_pack_against_oracle(oracle_mod, one, 4096)
+    assert mover.n_buckets == 10 and stream.size == 10 * 4096
+
+
+# ------------------------------------------------------------------ config 0 and a small adversarial set, full compare
+
+
+def test_config0_full(oracle_mod):
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    mover, _, _ = G.check_pack_against_oracle(oracle_mod, state)
+    assert (mover.total_bytes, mover.n_buckets) == (25_790_464, 25)
+    for plane in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V):
+        exp = G.check_shard_against_oracle(oracle_mod, state, state.plane_indices(plane), cfg.shard_r, cfg.shard_D)
+        assert exp.size == 921_088 * 4
+
+
+def test_small_adversarial_full(oracle_mod):
+    # same recipe as config 4 (log-uniform sizes, mixed dtypes, 2-byte-granular addresses), scaled to
+    # what the oracle packs in seconds: several chunks per large tensor, many sub-vector tensors
+    specs = layouts.adversarial_specs(3000, max_log2=18)
+    state = layouts.materialize_adversarial(specs, "cuda")
+    G.check_pack_against_oracle(oracle_mod, state, 1 << 20)
+    for e in (4, 2, 8):
+        idx = state.elem_size_indices(e)
+        flat = np.concatenate([state.host_bytes(i) for i in idx])
+        parts = []
+        for r in range(0, 64):
+            ex = ShardExtractor([state.descs()[i] for i in idx], r, 64)
+            out = ex.alloc_out()
+            ex.extract(out)
+            parts.append(out.cpu().numpy())
+        assert np.array_equal(np.concatenate(parts), flat)            # exact union coverage
+        for r in (0, 17, 63):
+            G.check_shard_against_oracle(oracle_mod, state, idx, r, 64, out_misalign=2 * (r % 8))
+
+
+def test_shard_edge_cases(oracle_mod):
+    specs = layouts.odd_specs(3, n_tensors=12)
+    state = layouts.materialize_adversarial(specs, "cuda", seed=3)
+    for e in (2, 4, 8):
+        idx = state.elem_size_indices(e)
+        if not idx:
+            continue
+        n_elems = sum(state.specs[i].numel for i in idx)
+        for D in (1, 2, 3, n_elems, n_elems + 5):          # D > N gives empty shards
+            for r in sorted({0, D // 2, D - 1}):
+                G.check_shard_against_oracle(oracle_mod, state, idx, r, D, out_misalign=2 * (r % 3))
+
+
+@pytest.mark.parametrize("nbytes,B", [(1, 256), (7, 256), (8, 256), (15, 256), (16, 256), (17, 256), (255, 256),
+                                      (256, 256), (257, 256), (4099, 1024), (65536 + 3, 4096), (1 << 20, 1 << 20),
+                                      ((1 << 20) + 24, 1 << 19), (3 * (1 << 20) + 1001, 768 * 1024)])
+def test_checksum_ragged_inputs(oracle_mod, nbytes, B):
+    data = torch.randint(0, 256, (nbytes,), dtype=torch.uint8, device="cuda",
+                         generator=torch.Generator("cuda").manual_seed(nbytes))
+    nb = -(-nbytes // B)
+    out = torch.full((nb + 2,), -1, dtype=torch.int64, device="cuda")
+    binding.tm_checksum(data.data_ptr(), nbytes, B, out[1:].data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.u64(out[1:1 + nb]), oracle_mod.checksum(data.cpu().numpy(), B))
+    assert int(out[0]) == -1 and int(out[-1]) == -1
+
+
+def test_checksum_constant_words_on_device():
+    c, n = 0x3F8000003F800000, 1 << 17      # fp32 1.0 pairs; closed form c * n^2 mod 2^64
+    data = torch.ones(2 * n, dtype=torch.float32, device="cuda")
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    binding.tm_checksum(data.data_ptr(), 8 * n, 8 * n, out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert int(G.u64(out)[0]) == (c * n * n) % (1 << 64)
+
+
+# ------------------------------------------------------------------ failure reporting without faulting anything
+
+
+def test_corruption_is_detected_and_bad_arguments_are_refused(oracle_mod):
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    mover, buckets, cks = G.gpu_pack(state)
+    host = buckets.cpu()
+    host[3 * cfg.bucket_bytes + 12345] ^= 0x10             # flip one bit of the host copy
+    received = host.cuda()
+    again = mover.alloc_checksums()
+    mover.checksum(received, again)
+    torch.cuda.synchronize()
+    bad = np.flatnonzero(G.u64(again) != cks)
+    assert bad.tolist() == [3]
+    s = torch.cuda.current_stream().cuda_stream
+    launches = binding.tm_launch_count()
+    with pytest.raises(binding.TmError) as e:              # packed buffer too small
+        binding.tm_state_pack(mover.plan, buckets.data_ptr(), mover.total_bytes - 256, None, s)
+    assert e.value.status == binding.TM_ERR_CAPACITY
+    with pytest.raises(binding.TmError) as e:              # packed buffer overlaps a source tensor
+        t = state.tensors[0]
+        binding.tm_state_pack(mover.plan, t.data_ptr(), 1 << 40, None, s)
+    assert e.value.status == binding.TM_ERR_OVERLAP
+    with pytest.raises(binding.TmError) as e:              # misaligned packed buffer
+        binding.tm_state_unpack(mover.plan, buckets.data_ptr() + 16, mover.total_bytes, s)
+    assert e.value.status == binding.TM_ERR_ALIGN
+    dup = [state.descs()[0], state.descs()[0]]             # two unpack targets are the same tensor
+    m2 = RoleMover(dup, 1 << 20)
+    with pytest.raises(binding.TmError) as e:
+        m2.unpack(buckets)
+    assert e.value.status == binding.TM_ERR_OVERLAP
+    assert binding.tm_launch_count() == launches           # nothing was launched by the refused calls
+    torch.cuda.synchronize()
+
+
+def test_repeated_runs_are_identical():
+    specs = layouts.adversarial_specs(500, max_log2=16)
+    state = layouts.materialize_adversarial(specs, "cuda")
+    _, b1, c1 = G.gpu_pack(state, 1 << 18)
+    first = b1.clone()
+    _, b2, c2 = G.gpu_pack(state, 1 << 18)
+    assert torch.equal(first, b2) and np.array_equal(c1, c2)

@@ -1,0 +1,136 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports everything the header
+declares, plans layouts that agree with the oracle's independent arithmetic, and rejects bad
+arguments before anything could be launched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_12636_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+FAKE = 0x7F00_0000_0000  # plausible device address; never dereferenced on the host
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load_library()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "tm_state.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(tm_[a-z_0-9]+)\s*\(", header))
+    assert declared == set(binding.SIGNATURES), declared ^ set(binding.SIGNATURES)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert lib.tm_strerror(0) == b"ok" and lib.tm_strerror(-8) == b"bounded device wait expired"
+
+
+def _descs(sizes, elem=2, base=FAKE, stride=1 << 24):
+    return [(base + k * stride, n, elem, 0) for k, n in enumerate(sizes)]
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_plan_layout_matches_oracle(lib, oracle_mod, seed):
+    rng = np.random.default_rng(seed)
+    sizes = [2 * int(rng.integers(1, 200_000)) for _ in range(int(rng.integers(1, 50)))]
+    B = 256 * int(rng.integers(1, 600))
+    plan = binding.Plan(_descs(sizes), B)
+    off, T, nb = oracle_mod.layout(sizes, B)
+    assert plan.offsets() == [int(x) for x in off]
+    assert (plan.total_bytes, plan.n_buckets) == (T, nb)
+    assert plan.workspace_bytes % 256 == 0 and plan.workspace_bytes >= 512
+
+
+def test_plan_full_size_configs_match_oracle(lib, oracle_mod):
+    from paper_2412_12636_b200 import layouts
+    for idx in range(4):
+        cfg = layouts.role_config(idx)
+        sizes = [s.nbytes for s in cfg.specs()]
+        descs = []
+        addr = FAKE
+        for s in cfg.specs():
+            descs.append((addr, s.nbytes, s.elem_size, s.plane))
+            addr += (s.nbytes + 511) // 512 * 512
+        plan = binding.Plan(descs, cfg.bucket_bytes)
+        off, T, nb = oracle_mod.layout(sizes, cfg.bucket_bytes)
+        assert plan.offsets() == [int(x) for x in off] and (plan.total_bytes, plan.n_buckets) == (T, nb)
+
+
+def test_plan_rejects_bad_arguments(lib):
+    cases = [
+        ([(FAKE, 4, 2, 0)], 100, binding.TM_ERR_ALIGN),       # bucket not a multiple of 256
+        ([(FAKE, 4, 2, 0)], 0, binding.TM_ERR_ARG),
+        ([(FAKE, 4, 2, 0)], (1 << 35) + 256, binding.TM_ERR_ARG),
+        ([(FAKE + 1, 4, 2, 0)], 256, binding.TM_ERR_ALIGN),   # odd address
+        ([(FAKE, 0, 2, 0)], 256, binding.TM_ERR_ARG),
+        ([(FAKE, 6, 4, 0)], 256, binding.TM_ERR_ARG),         # not a whole number of elements
+        ([(FAKE, 6, 3, 0)], 256, binding.TM_ERR_DTYPE),
+        ([(0, 4, 2, 0)], 256, binding.TM_ERR_ARG),
+        ([], 256, binding.TM_ERR_ARG),
+    ]
+    for descs, B, code in cases:
+        with pytest.raises(binding.TmError) as e:
+            binding.Plan(descs, B)
+        assert e.value.status == code, (descs, B)
+
+
+def test_ops_refuse_a_plan_without_work_list(lib):
+    plan = binding.Plan(_descs([512, 1024]), 256)
+    for call in (lambda: binding.tm_state_pack(plan, FAKE + (1 << 30), 1 << 20, None, 0),
+                 lambda: binding.tm_state_unpack(plan, FAKE + (1 << 30), 1 << 20, 0)):
+        with pytest.raises(binding.TmError) as e:
+            call()
+        assert e.value.status == binding.TM_ERR_STATE
+
+
+def test_shard_bounds_and_validation(lib):
+    for N, D in ((10, 3), (1069711360, 24), (1, 64), ((1 << 64) - 1, (1 << 32) - 1)):
+        for r in sorted({0, 1 % D, D // 2, D - 1}):
+            assert binding.tm_shard_bounds(N, r, D) == ((r * N) // D, ((r + 1) * N) // D)
+    for r, D in ((2, 2), (0, 0)):
+        with pytest.raises(binding.TmError) as e:
+            binding.tm_shard_bounds(10, r, D)
+        assert e.value.status == binding.TM_ERR_RANK
+    mixed = [(FAKE, 8, 4, 1), (FAKE + 4096, 8, 2, 0)]
+    with pytest.raises(binding.TmError) as e:
+        binding.tm_shard_workspace(mixed, 0, 2)
+    assert e.value.status == binding.TM_ERR_DTYPE
+    with pytest.raises(binding.TmError) as e:
+        binding.tm_shard_workspace(_descs([8, 8], elem=4), 3, 2)
+    assert e.value.status == binding.TM_ERR_RANK
+    assert binding.tm_shard_workspace(_descs([1 << 20, 1 << 20], elem=4), 1, 2) >= 512
+    # argument errors are reported before any device work
+    with pytest.raises(binding.TmError) as e:
+        binding.tm_shard_extract(_descs([1 << 20], elem=4), 0, 1, FAKE + 4096, 1 << 20, FAKE + (1 << 30), 1 << 20, 0)
+    assert e.value.status == binding.TM_ERR_OVERLAP
+    with pytest.raises(binding.TmError) as e:
+        binding.tm_shard_extract(_descs([1 << 20], elem=4), 0, 1, FAKE + (1 << 28), 100, FAKE + (1 << 30), 1 << 20, 0)
+    assert e.value.status == binding.TM_ERR_CAPACITY
+
+
+def test_checksum_argument_validation(lib):
+    for args, code in (((FAKE, 1024, 100, FAKE + 4096, 0), binding.TM_ERR_ALIGN),
+                       ((FAKE, 1024, 0, FAKE + 4096, 0), binding.TM_ERR_ARG),
+                       ((FAKE + 8, 1024, 256, FAKE + 4096, 0), binding.TM_ERR_ALIGN),
+                       ((FAKE, 1024, 256, None, 0), binding.TM_ERR_ARG)):
+        with pytest.raises(binding.TmError) as e:
+            binding.tm_checksum(*args)
+        assert e.value.status == code
+    binding.tm_checksum(FAKE, 0, 256, None, 0)   # empty input: nothing to do
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="only meaningful on a machine without a GPU")
+def test_no_cpu_fallback_without_a_gpu(lib):
+    host = np.zeros(1024, dtype=np.uint8)
+    out = np.zeros(4, dtype=np.uint64)
+    before = binding.tm_launch_count()
+    with pytest.raises(binding.TmError) as e:
+        binding.tm_checksum(host.ctypes.data & ~15, 512, 256, out.ctypes.data, 0)
+    assert e.value.status == binding.TM_ERR_CUDA
+    assert binding.tm_launch_count() == before and not out.any()
