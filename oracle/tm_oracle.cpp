@@ -141,11 +141,12 @@ int oracle_pack_range(const uint8_t* const* ptrs, const uint64_t* nbytes, uint64
   uint64_t pos = 0;
   for (uint64_t k = 0; k < n; ++k) {
     pos = round_up_256(pos);
-    for (uint64_t j = 0; j < nbytes[k]; ++j) {
-      uint64_t s = pos + j;
-      if (s >= lo && s < hi) {
-        if (ptrs[k] == NULL) return ORC_ERR_ARG;
-        out[s - lo] = ptrs[k][j];
+    bool intersects = (pos < hi) && (pos + nbytes[k] > lo);  // tensors wholly outside are skipped
+    if (intersects) {
+      if (ptrs[k] == NULL) return ORC_ERR_ARG;
+      for (uint64_t j = 0; j < nbytes[k]; ++j) {
+        uint64_t s = pos + j;
+        if (s >= lo && s < hi) out[s - lo] = ptrs[k][j];
       }
     }
     pos += nbytes[k];

@@ -1,0 +1,76 @@
+"""The N > 1 path of the benchmark on CPU: ranks are independent replicas, so the only cross-rank
+logic is the aggregation (slowest rank's device time, sum of bytes).  Run with gloo, world size 2."""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = r"""
+import os, sys, json
+sys.path.insert(0, os.environ["TM_ROOT"])
+import torch.distributed as dist
+import bench
+dist.init_process_group("gloo")
+rank = dist.get_rank()
+ms, nbytes = bench.aggregate_over_ranks(10.0 + 5.0 * rank, 1000 * (rank + 1))
+dist.barrier()
+print(json.dumps({"rank": rank, "ms": ms, "bytes": nbytes}))
+dist.destroy_process_group()
+"""
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def test_aggregate_over_two_gloo_ranks(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER)
+    port = _free_port()
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, TM_ROOT=ROOT, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        out, err = p.communicate(timeout=120)
+        assert p.returncode == 0, err[-2000:]
+        outs.append(json.loads(out.strip().splitlines()[-1]))
+    for o in outs:
+        assert o["ms"] == 15.0 and o["bytes"] == 3000      # max over ranks, sum over ranks
+
+
+def test_single_process_aggregate_and_byte_accounting():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.aggregate_over_ranks(7.5, 123) == (7.5, 123)
+    b = bench.step_bytes(state_bytes=1400, total_bytes=1536, n_buckets=2, shard_bytes=[100, 100, 100])
+    assert b == {"pack": 1400 + 1536 + 16, "checksum": 1536 + 16, "unpack": 2800, "shard": 600}
+    assert abs(bench.gbs(2e9, 1000.0) - 2.0) < 1e-12
+    s = bench.ClockSampler.summarise(["1965, 1965, Not Active, Not Active, Not Active, Active",
+                                      "1800, 1965, Not Active, Not Active, Not Active, Not Active", "garbage"])
+    assert s["sm_mhz"] == 1882.5 and s["sm_max_mhz"] == 1965.0 and s["reasons"] == ["sw_power_cap"]
+
+
+def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
+    env = dict(os.environ)
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg0",
+                          "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
+    env["RANK"] = "1"
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg0"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and out.stdout.strip() == ""
