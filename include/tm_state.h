@@ -156,6 +156,27 @@ int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, ui
                      void* d_out, uint64_t out_capacity, uint64_t* out_elems,
                      void* d_workspace, uint64_t workspace_bytes, void* stream);
 
+/* Size of the library-resident scratch array used by tm_shard_extract_static. */
+#define TM_STATIC_SCRATCH_BYTES (1u << 20)
+
+/* Shard extract without caller scratch.  (The paper has no counterpart: this entry point exists
+ * for the library's users, not for the method.)  It is for callers that are handed tensors but
+ * cannot allocate on the device: a recovery hook running while the framework's allocator owns the
+ * whole GPU, code that must avoid cudaMalloc because it synchronises the device and can fail when
+ * memory is full, or a plugin with no allocator.  Same arguments, checks, results and errors as
+ * tm_shard_extract, minus the workspace: the work list goes into a fixed array of
+ * TM_STATIC_SCRATCH_BYTES (1 MiB) of device global memory that is part of the library image; every
+ * GPU that loads the library holds that array until the process exits.  A shard whose list does
+ * not fit (with the default 64 KiB pieces: more than about 1.8 GiB of output, or more than about
+ * 29 000 tensor pieces) is refused with TM_ERR_CAPACITY and nothing is launched.  The call makes no
+ * device allocation and frees none.  The first call on each GPU resolves the array's device address
+ * once, with that GPU current; make that call before starting any stream capture.  All calls on a
+ * GPU share the array, which keeps the previous call's contents: the part that must start from zero
+ * (the status block) is cleared on every call, and calls whose device work can overlap in time (two
+ * streams, two threads) race on the list — serialise them on one stream. */
+int tm_shard_extract_static(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                            void* d_out, uint64_t out_capacity, uint64_t* out_elems, void* stream);
+
 /* Status word of a raw workspace used by tm_shard_extract (same meaning as tm_plan_status). */
 int tm_workspace_status(const void* d_workspace, void* stream, int* device_status);
 

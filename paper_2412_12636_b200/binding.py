@@ -32,6 +32,7 @@ SIGNATURES = {
     "tm_shard_bounds": (_int, [_u64, _u32, _u32, _p, _p]),
     "tm_shard_workspace": (_int, [_p, _u64, _u32, _u32, _p]),
     "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
+    "tm_shard_extract_static": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p]),
     "tm_workspace_status": (_int, [_p, _p, _p]),
     "tm_checksum": (_int, [_p, _u64, _u64, _p, _p]),
     "tm_strerror": (ctypes.c_char_p, [_int]),
@@ -157,6 +158,16 @@ def tm_shard_extract(descs, r: int, D: int, d_out: int, out_capacity: int, d_wor
     n = _u64()
     _check(load_library().tm_shard_extract(arr, len(arr), r, D, d_out, out_capacity, ctypes.byref(n),
                                            d_workspace, workspace_bytes, stream), "tm_shard_extract")
+    return n.value
+
+
+def tm_shard_extract_static(descs, r: int, D: int, d_out: int, out_capacity: int, stream: int) -> int:
+    """Shard extract that uses the library's own fixed device scratch (no workspace argument, no
+    device allocation); for callers that cannot allocate.  Returns the number of elements written."""
+    arr = descs if isinstance(descs, ctypes.Array) else make_descs(descs)
+    n = _u64()
+    _check(load_library().tm_shard_extract_static(arr, len(arr), r, D, d_out, out_capacity, ctypes.byref(n),
+                                                  stream), "tm_shard_extract_static")
     return n.value
 
 

@@ -1,0 +1,105 @@
+// Shard extract for callers that cannot allocate device memory.
+//
+// tm_shard_extract needs a small device-resident work list and asks its caller for the scratch to
+// hold it.  Some callers have no way to provide that: a recovery hook that runs while the training
+// framework's caching allocator already owns the whole GPU, a handler that must not call cudaMalloc
+// because that call synchronises the device and may fail exactly when memory is exhausted, or a
+// plugin that is handed tensors but no allocator.  For them this file keeps the scratch inside the
+// library itself, as a fixed array in device global memory, and exports one extra entry point.
+//
+// Rules that follow from that choice:
+//   * the array is TM_STATIC_SCRATCH_BYTES long on every GPU whose context loads this library and
+//     stays resident until the process exits;
+//   * a request whose work list does not fit is refused with TM_ERR_CAPACITY, nothing is launched;
+//   * all calls on one GPU share the one array and it still holds the previous call's list, so the
+//     status block is cleared on every call and two calls whose device work may overlap (different
+//     streams, or one stream per thread) would overwrite each other's list: issue them on one stream;
+//   * the first call on each GPU looks up the array's device address (cudaGetSymbolAddress) with that
+//     GPU current; make that first call outside any stream capture.
+// No cudaMalloc, cudaFree or other allocating routine is called here.
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "tm_internal.h"
+
+int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
+int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                      uint32_t* elem_size, uint64_t* n_elems);
+void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
+                       uint64_t d_out, tms::WorkList* wl);
+
+// In host code this name is only a handle for the runtime, not a device address: never pass it to a
+// kernel.  The address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[TM_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_mutex;
+uint8_t* g_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device; looked up once per device.
+cudaError_t scratch_for_current_device(uint8_t** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (g_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_addr[dev] = static_cast<uint8_t*>(p);
+  }
+  *out = g_scratch_addr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int tm_shard_extract_static(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                                       void* d_out, uint64_t out_capacity, uint64_t* out_elems,
+                                       void* stream) {
+  uint32_t e = 0;
+  uint64_t n_elems = 0;
+  int rc = tm_shard_validate(plane_descs, n_desc, r, D, &e, &n_elems);
+  if (rc != TM_OK) return rc;
+  uint64_t lo = 0, hi = 0;
+  rc = tm_bounds_u128(n_elems, r, D, &lo, &hi);
+  if (rc != TM_OK) return rc;
+  if (out_elems != nullptr) *out_elems = hi - lo;
+  if (hi == lo) return TM_OK;
+  if (d_out == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_out & 1) != 0) return TM_ERR_ALIGN;
+  const uint64_t out_bytes = (hi - lo) * e;
+  if (out_capacity < out_bytes) return TM_ERR_CAPACITY;
+  // refuse oversized requests from the byte count alone, before building any list
+  const uint64_t chunk = tms::tuning().chunk_bytes;
+  const uint64_t min_segs = out_bytes / chunk;
+  if (tms::workspace_layout(min_segs, 1).total > TM_STATIC_SCRATCH_BYTES) return TM_ERR_CAPACITY;
+  const uint64_t out_addr = (uint64_t)(uintptr_t)d_out;
+  for (uint64_t k = 0; k < n_desc; ++k) {
+    const uint64_t a = (uint64_t)(uintptr_t)plane_descs[k].ptr;
+    if (a < out_addr + out_bytes && out_addr < a + plane_descs[k].nbytes) return TM_ERR_OVERLAP;
+  }
+  tms::WorkList wl;
+  tm_shard_worklist(plane_descs, n_desc, e, lo, hi, out_addr, &wl);
+  const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
+  if (l.total > TM_STATIC_SCRATCH_BYTES) return TM_ERR_CAPACITY;
+
+  uint8_t* scratch = nullptr;
+  cudaError_t ce = scratch_for_current_device(&scratch);
+  if (ce != cudaSuccess) return TM_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  // the array still holds the previous call's status block and list: clear the former, overwrite the latter
+  if ((ce = cudaMemsetAsync(scratch, 0, tms::kStatusBlockBytes, st)) != cudaSuccess) return TM_ERR_CUDA;
+  if ((ce = cudaMemcpyAsync(scratch + l.segs_off, wl.segs.data(), wl.segs.size() * sizeof(tms::Seg),
+                            cudaMemcpyHostToDevice, st)) != cudaSuccess) return TM_ERR_CUDA;
+  if ((ce = cudaMemcpyAsync(scratch + l.items_off, wl.item_first.data(), wl.item_first.size() * sizeof(uint32_t),
+                            cudaMemcpyHostToDevice, st)) != cudaSuccess) return TM_ERR_CUDA;
+  const int err = tms::launch_copy((const tms::Seg*)(scratch + l.segs_off), (const uint32_t*)(scratch + l.items_off),
+                                   (uint32_t)wl.n_items(), (uint8_t*)d_out, /*to_tensors=*/false,
+                                   (int*)scratch, stream);
+  return err == 0 ? TM_OK : TM_ERR_CUDA;
+}
