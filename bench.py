@@ -306,7 +306,8 @@ def run_ours(args) -> None:
     e2e = None
     cpu_baseline = None
     if rank == 0 and world == 1:
-        e2e = run_e2e(args, cfg, state, mover, buckets, cks_fused, bytes_per_step, one_step, shards)
+        if not args.no_e2e:
+            e2e = run_e2e(args, cfg, state, mover, buckets, cks_fused, bytes_per_step, one_step, shards)
         if not args.no_cpu_baseline:
             step, sample = oracle_sample_step(cfg)
             dt, nb = step()
@@ -399,6 +400,7 @@ def main() -> None:
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler launch lists)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -110,8 +110,18 @@ def _llama_model(layers: int, h: int, q_out: int, kv_out: int, ffn: int, vocab_r
 MiB = 1 << 20
 
 
-def role_config(index: int) -> RoleConfig:
-    """The four model-shaped role layouts (config 4, the adversarial set, is `adversarial_specs`)."""
+def role_config(index: int, layers: Optional[int] = None) -> RoleConfig:
+    """The four model-shaped role layouts (config 4, the adversarial set, is `adversarial_specs`).
+    `layers` overrides the number of transformer layers (reduced cases for profiling)."""
+    if layers is not None:
+        full = role_config(index)
+        assert 0 < layers <= {0: 2, 1: 22, 2: 32, 3: 10}[index]
+
+        def layer_of(name: str) -> int:
+            head = name.split(".")[0]
+            return int(head[1:]) if head[0] == "l" and head[1:].isdigit() else -1
+        keep = tuple(t for t in full.model if layer_of(t[0]) < layers)
+        return dataclasses.replace(full, name=f"{full.name}-{layers}layers", model=keep)
     if index == 0:   # tiny GPT, TP=1 PP=1 DP=2
         return RoleConfig(0, "tiny-gpt", 0, 1 * MiB, 1, 2, _gpt_model(2, 256, 1024, 1024))
     if index == 1:   # Llama-style 1.1B, TP=1 PP=1; 32 heads / 4 KV heads, head dim 64
