@@ -162,3 +162,80 @@ def test_adversarial_20000_tensors_single_launch(oracle_mod):
         check_shard_sampled(oracle_mod, state, idx, r, 64)
     for e in (2, 8):                                     # generalisation: other element sizes
         check_shard_sampled(oracle_mod, state, state.elem_size_indices(e), 13, 64)
+
+
+def test_adversarial_200000_tensors_in_waves(oracle_mod):
+    """Config 4 as specified: 200 000 tensors, about 257 GB of state — more than one GPU holds next
+    to its packed copy.  Processed in waves that each cover whole buckets of the complete stream."""
+    from paper_2412_12636_b200 import waves
+    specs = layouts.adversarial_specs(200_000)
+    sizes = [s.nbytes for s in specs]
+    B = layouts.ADVERSARIAL_BUCKET
+    fake = 0x7F00_0000_0000          # host-only plan: layout of the complete list, nothing is launched
+    plan = binding.Plan([(fake, n, s.elem_size, s.plane) for n, s in zip(sizes, specs)], B)
+    off, T, nb = oracle_mod.layout(sizes, B)
+    off = [int(x) for x in off]
+    assert plan.offsets() == off and (plan.total_bytes, plan.n_buckets) == (T, nb)
+    del plan
+    # shard bounds of the complete fp32 plane tile [0, N) exactly (offsets only, no data)
+    N = sum(s.numel for s in specs if s.elem_size == 4)
+    prev = 0
+    for r in range(64):
+        lo, hi = binding.tm_shard_bounds(N, r, 64)
+        assert (lo, hi) == oracle_mod.shard_bounds(N, r, 64) and lo == prev
+        prev = hi
+    assert prev == N
+
+    ws = waves.cut_waves(sizes, off, T, B, budget_bytes=24 << 30)
+    assert ws[0].stream_begin == 0 and ws[-1].stream_end == T and sum(w.n_buckets for w in ws) == nb
+    all_cks = []
+    for wi, w in enumerate(ws):
+        wave_specs = [specs[p.tensor] for p in w.parts]
+        full = layouts.materialize_adversarial(wave_specs, "cuda", wave=wi)
+        part_specs, part_tensors = [], []
+        for p, s, t in zip(w.parts, wave_specs, full.tensors):
+            part_specs.append(layouts.TensorSpec(s.name, p.nbytes // s.elem_size, s.dtype, s.plane, s.model_index))
+            part_tensors.append(t[p.byte_start:p.byte_start + p.nbytes])
+        state = layouts.RoleState(f"wave{wi}", part_specs, part_tensors, B, 0, 64, full.arena)
+        mover, buckets, cks = G.gpu_pack(state, B)
+        assert mover.total_bytes == w.stream_end - w.stream_begin and mover.n_buckets == w.n_buckets
+        alone = mover.alloc_checksums()
+        mover.checksum(buckets, alone)
+        torch.cuda.synchronize()
+        assert np.array_equal(G.u64(alone), cks)
+        all_cks.append(cks)
+        rng = np.random.default_rng(100 + wi)
+        sample = sorted({0, mover.n_buckets - 1, int(rng.integers(0, mover.n_buckets))})
+        woff = check_sampled_buckets(oracle_mod, state, mover, buckets, cks, sample)
+        check_stream_structure_on_device(state, woff, buckets, mover.total_bytes)
+        for a, b in zip(state.tensors, check_unpack_parts(state, buckets, B)):
+            assert torch.equal(a, b)
+        del buckets, alone
+        idx = state.elem_size_indices(4)
+        if idx:
+            descs = [state.descs()[i] for i in idx]
+            flat = torch.cat([state.tensors[i] for i in idx])
+            parts = []
+            for r in range(64):
+                ex = ShardExtractor(descs, r, 64)
+                out = ex.alloc_out()
+                ex.extract(out)
+                parts.append(out)
+            torch.cuda.synchronize()
+            assert torch.equal(torch.cat(parts), flat)
+            del parts, flat
+            check_shard_sampled(oracle_mod, state, idx, int(rng.integers(0, 64)), 64)
+        del state, full, mover
+        torch.cuda.empty_cache()
+    assert sum(c.size for c in all_cks) == nb
+
+
+def check_unpack_parts(state, buckets, B):
+    """Unpack into fresh 0xA5-filled buffers, one per tensor part; returns them."""
+    targets = [torch.full((t.numel(),), 0xA5, dtype=torch.uint8, device="cuda") for t in state.tensors]
+    descs = [(t.data_ptr(), s.nbytes, s.elem_size, s.plane) for t, s in zip(targets, state.specs)]
+    um = RoleMover(descs, B)
+    um.unpack(buckets)
+    torch.cuda.synchronize()
+    assert um.status() == 0
+    return targets
