@@ -77,7 +77,8 @@ def gbs(nbytes: float, ms: float) -> float:
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    """Samples SM clock and throttle reasons of one GPU while a region runs: NVML polled every
+    20 ms from a thread (read-only queries), or `nvidia-smi -lms 100` when NVML is not importable."""
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -86,8 +87,46 @@ class ClockSampler:
         self.proc: Optional[subprocess.Popen] = None
         self.lines: List[str] = []
         self.thread: Optional[threading.Thread] = None
+        self._stop = threading.Event()
+        self._nvml = None
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        try:
+            uuid = str(torch.cuda.get_device_properties(self.gpu_index).uuid)
+            h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode() if not uuid.startswith("GPU-") else uuid.encode())
+        except Exception:
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.gpu_index)
+        return pynvml, h
 
     def start(self) -> None:
+        try:
+            nv, h = self._nvml_handle()
+            mx = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            bits = [(getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8), "hw"),
+                    (getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40), "hwt"),
+                    (getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20), "swt"),
+                    (getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4), "pc")]
+            get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                nv.nvmlDeviceGetCurrentClocksThrottleReasons
+
+            def poll():
+                while not self._stop.is_set():
+                    try:
+                        mhz = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+                        r = get_reasons(h)
+                        flags = ["Active" if (r & bit) else "Not Active" for bit, _ in bits]
+                        self.lines.append(f"{mhz}, {mx}, " + ", ".join(flags))
+                    except Exception:
+                        pass
+                    self._stop.wait(0.02)
+            self._nvml = nv
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self._nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
@@ -95,6 +134,7 @@ class ClockSampler:
         except Exception:
             self.proc = None
             return
+
         def pump():
             for line in self.proc.stdout:
                 self.lines.append(line.strip())
@@ -102,6 +142,12 @@ class ClockSampler:
         self.thread.start()
 
     def stop(self) -> Dict[str, object]:
+        if self._nvml is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+            out = self.summarise(self.lines)
+            out["source"] = "nvml"
+            return out
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -111,7 +157,9 @@ class ClockSampler:
             self.proc.kill()
         if self.thread is not None:
             self.thread.join(timeout=2)
-        return self.summarise(self.lines)
+        out = self.summarise(self.lines)
+        out["source"] = "nvidia-smi"
+        return out
 
     @staticmethod
     def summarise(lines: List[str]) -> Dict[str, object]:
@@ -231,7 +279,7 @@ def run_ours(args) -> None:
     cks_alone = mover.alloc_checksums()
     shards = []
     for plane in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V):
-        ex = ShardExtractor([target.descs()[i] for i in target.plane_indices(plane)], cfg.shard_r, cfg.shard_D)
+        ex = ShardExtractor(target.descs_of(target.plane_indices(plane)), cfg.shard_r, cfg.shard_D)
         shards.append((ex, ex.alloc_out()))
     per_op = step_bytes(state.state_bytes, mover.total_bytes, mover.n_buckets, [ex.out_bytes for ex, _ in shards])
     bytes_per_step = sum(per_op.values())

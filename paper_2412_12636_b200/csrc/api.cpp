@@ -118,7 +118,8 @@ int tm_state_pack(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint6
   if (d_checksums != nullptr)
     TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), st));
   const uint8_t* ws = plan->d_workspace;
-  int e = tms::launch_pack((const tms::Seg*)(ws + plan->ws_layout.segs_off),
+  auto pack_fn = tms::tuning().use_ring ? tms::launch_pack_ring : tms::launch_pack;
+  int e = pack_fn((const tms::Seg*)(ws + plan->ws_layout.segs_off),
                           (const uint32_t*)(ws + plan->ws_layout.items_off),
                           (uint32_t)plan->work.n_items(), (uint8_t*)d_buckets,
                           (unsigned long long*)d_checksums, (int*)plan->d_workspace, stream);
@@ -136,7 +137,8 @@ int tm_state_unpack(const tm_plan* plan, const void* d_buckets, uint64_t nbytes,
   if (plan->targets_disjoint == 0) plan->targets_disjoint = tm_targets_disjoint(plan);
   if (plan->targets_disjoint < 0) return TM_ERR_OVERLAP;
   const uint8_t* ws = plan->d_workspace;
-  int e = tms::launch_copy((const tms::Seg*)(ws + plan->ws_layout.segs_off),
+  auto copy_fn = tms::tuning().use_ring ? tms::launch_copy_ring : tms::launch_copy;
+  int e = copy_fn((const tms::Seg*)(ws + plan->ws_layout.segs_off),
                           (const uint32_t*)(ws + plan->ws_layout.items_off),
                           (uint32_t)plan->work.n_items(), (uint8_t*)const_cast<void*>(d_buckets),
                           /*to_tensors=*/true, (int*)plan->d_workspace, stream);
@@ -192,7 +194,8 @@ int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, ui
   rc = upload_worklist(wl, l, (uint8_t*)d_workspace, (cudaStream_t)stream);
   if (rc != TM_OK) return rc;
   const uint8_t* ws = (const uint8_t*)d_workspace;
-  int err = tms::launch_copy((const tms::Seg*)(ws + l.segs_off), (const uint32_t*)(ws + l.items_off),
+  auto copy_fn = tms::tuning().use_ring ? tms::launch_copy_ring : tms::launch_copy;
+  int err = copy_fn((const tms::Seg*)(ws + l.segs_off), (const uint32_t*)(ws + l.items_off),
                             (uint32_t)wl.n_items(), (uint8_t*)d_out, /*to_tensors=*/false,
                             (int*)d_workspace, stream);
   return err == 0 ? TM_OK : cuda_fail(err);

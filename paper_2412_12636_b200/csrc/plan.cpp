@@ -27,6 +27,9 @@ const Tuning& tuning() {
     x.group_bytes = env_u64("TM_GROUP_BYTES", 64 * 1024);
     x.group_max = (uint32_t)env_u64("TM_GROUP_MAX", 64);
     x.ctas_per_sm = (uint32_t)env_u64("TM_CTAS_PER_SM", 4);
+    x.ring_ctas_per_sm = (uint32_t)env_u64("TM_RING_CTAS_PER_SM", 1);
+    const char* ring = std::getenv("TM_USE_RING");
+    x.use_ring = !(ring != nullptr && ring[0] == '0');
     return x;
   }();
   return t;

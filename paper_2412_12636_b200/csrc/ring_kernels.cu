@@ -1,0 +1,401 @@
+// Bulk-copy ("TMA") ring kernels for sm_100a: the same pack / copy work as kernels.cu, but large
+// pieces travel global -> shared memory with cp.async.bulk issued by one producer thread into a
+// ring of stages guarded by mbarriers.  When source and destination are both 16-byte aligned the
+// stage goes straight back out, shared memory -> global, with a bulk store issued by one store
+// thread, and the eight consumer warps only read the stage to accumulate the checksum.  When the
+// source sits at a 2-byte-granular address the consumers re-align the stage in registers and write
+// 16-byte vectors themselves.  The producer runs ahead across piece and item boundaries, so the
+// loads of the next pieces are in flight while the current one is consumed.
+//
+// Misaligned sources cost no extra global traffic here: the producer fetches the aligned superset
+// of the source span (one extra 16-byte vector per stage) and the consumers shift in registers.
+// The superset stays inside 16-byte lines that hold at least one byte of the tensor.
+//
+// Every wait is bounded in time.  If one expires the waiter records TM_ERR_TIMEOUT in the status
+// word, raises a block-wide abort flag that all roles poll, and the producer waits (bounded) for its
+// own copies in flight before the block exits; the context stays usable.
+//
+// Small pieces (items that group several pieces, or single pieces below kBulkMinVectors) are
+// copied by the consumer warps with the register routines of device_util.cuh.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "device_util.cuh"
+#include "tm_internal.h"
+
+namespace tms {
+
+constexpr int kRingStages = 3;
+constexpr uint32_t kStageBytes = 32 * 1024;
+constexpr uint32_t kStageVectors = kStageBytes / 16;
+constexpr int kConsWarps = 8;
+constexpr int kConsThreads = kConsWarps * 32;
+constexpr int kRingThreads = kConsThreads + 64;     // + one producer warp + one store warp
+constexpr uint32_t kBulkMinVectors = 128;           // pieces below 2 KiB are not worth a stage
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(b)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase with the given parity; gives up after kWaitLimitNs or when the block aborts.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(b, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try(b, parity)) return true;
+    if (*abort_flag != 0) return false;
+    if (global_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+// Non-multicast 1-D bulk copy global -> this block's shared memory, completion on an mbarrier.
+__device__ __forceinline__ void bulk_g2s(void* smem, const void* g, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem)),
+               "l"(g), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Bulk store this block's shared memory -> global, tracked by the issuing thread's bulk groups.
+__device__ __forceinline__ void bulk_s2g(void* g, const void* smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(g), "r"(smem_u32(smem)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until all but the newest N bulk stores of this thread have finished READING shared memory.
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void consumer_barrier() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory");
+}
+
+// How one piece is cut into ring stages.  Destination vectors are 16-byte aligned; `head` bytes
+// before the first aligned destination vector and `rem` bytes after the last full one are copied
+// directly.  Stage t carries destination vectors [t*V, t*V + cnt) and is loaded from the aligned
+// source address sa + 16*t*V, (cnt + extra) vectors long, extra = 1 when the source is shifted.
+struct BulkPlan {
+  const uint8_t* src;   // after the head
+  uint8_t* dst;         // after the head, 16-byte aligned
+  const uint8_t* sa;    // src rounded down to 16 bytes
+  uint32_t a;           // src - sa, even, 0..14
+  uint32_t head, nfull, rem, V, ntiles;
+  bool straight;        // source and destination both aligned: stages are stored back by bulk stores
+};
+
+template <bool TO_TENSORS>
+__device__ __forceinline__ bool plan_bulk(const Seg& s, uint8_t* flat, BulkPlan& p) {
+  uint8_t* tensor = reinterpret_cast<uint8_t*>(s.tensor);
+  uint8_t* f = flat + s.off;
+  const uint8_t* src = TO_TENSORS ? f : tensor;
+  uint8_t* dst = TO_TENSORS ? tensor : f;
+  uint32_t n = s.nbytes;
+  uint32_t head = (uint32_t)((0 - (uintptr_t)dst) & 15);
+  if (head > n) head = n;
+  p.head = head;
+  p.src = src + head;
+  p.dst = dst + head;
+  n -= head;
+  p.nfull = n >> 4;
+  p.rem = n & 15;
+  p.a = (uint32_t)((uintptr_t)p.src & 15);
+  p.sa = p.src - p.a;
+  p.V = kStageVectors - (p.a != 0 ? 1u : 0u);
+  p.ntiles = (p.nfull + p.V - 1) / p.V;
+  p.straight = (p.a == 0);   // the destination is aligned by construction (head bytes are cut off)
+  return p.nfull >= kBulkMinVectors;
+}
+
+struct RingShared {
+  uint64_t full[kRingStages];
+  uint64_t empty[kRingStages];
+  unsigned long long red[kConsWarps];
+  int abort_flag;
+};
+
+__device__ __forceinline__ void raise_timeout(int* status, RingShared* sh) {
+  if (status != nullptr) atomicExch(status, (int)TM_ERR_TIMEOUT);
+  atomicExch(&sh->abort_flag, 1);
+}
+
+// Sum over the consumer warps of a per-thread value, added to *target by one thread.
+__device__ __forceinline__ void consumer_flush(u64 value, u64* target, RingShared* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) value += __shfl_xor_sync(0xffffffffu, value, o);
+  if ((threadIdx.x & 31) == 0) sh->red[threadIdx.x >> 5] = value;
+  consumer_barrier();
+  if (threadIdx.x == 0) {
+    u64 total = 0;
+#pragma unroll
+    for (int w = 0; w < kConsWarps; ++w) total += sh->red[w];
+    if (total != 0) atomicAdd(target, total);
+  }
+  consumer_barrier();
+}
+
+// PACK: tensors -> stream with padding and checksums.  Otherwise a plain copy of pieces, direction
+// given by TO_TENSORS (PACK implies TO_TENSORS == false).
+template <bool PACK, bool TO_TENSORS>
+__global__ void __launch_bounds__(kRingThreads, 1)
+ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
+            uint8_t* __restrict__ flat, u64* __restrict__ checksums, int* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t ring[];
+  __shared__ RingShared sh;
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRingStages; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], kConsWarps + 1);   // consumer warps + the store thread
+    }
+    sh.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int* abort_flag = &sh.abort_flag;
+
+  if (warp == kConsWarps) {
+    // ---------------- producer: one thread issues every bulk load of this block, in item order
+    if (lane != 0) return;
+    uint32_t stage = 0, phase = 0, issued = 0;
+    bool ok = true;
+    for (uint32_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+      const uint32_t first = item_first[item];
+      if (item_first[item + 1] - first != 1) continue;
+      const Seg s = segs[first];
+      BulkPlan p;
+      if (!plan_bulk<TO_TENSORS>(s, flat, p)) continue;
+      const uint32_t extra = p.a != 0 ? 1u : 0u;
+      for (uint32_t t = 0; t < p.ntiles; ++t) {
+        if (!mbar_wait(&sh.empty[stage], phase ^ 1u, abort_flag)) {
+          raise_timeout(status, &sh);
+          ok = false;
+          break;
+        }
+        uint32_t cnt = p.nfull - t * p.V;
+        if (cnt > p.V) cnt = p.V;
+        const uint32_t bytes = (cnt + extra) * 16u;
+        mbar_expect_tx(&sh.full[stage], bytes);
+        bulk_g2s(ring + (size_t)stage * kStageBytes, p.sa + (size_t)t * p.V * 16u, bytes, &sh.full[stage]);
+        ++issued;
+        if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok || *abort_flag != 0) {
+      // leave no copy in flight: the latest load of each stage must have landed before the block exits
+      uint32_t n = issued < (uint32_t)kRingStages ? issued : (uint32_t)kRingStages;
+      uint32_t st = stage, ph = phase;
+      for (uint32_t k = 0; k < n; ++k) {
+        if (st == 0) { st = kRingStages; ph ^= 1u; }
+        --st;
+        const unsigned long long t0 = global_ns();
+        while (!mbar_try(&sh.full[st], ph) && global_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+    return;
+  }
+
+  if (warp == kConsWarps + 1) {
+    // ---------------- store thread: sends aligned stages back out with bulk stores, in item order
+    if (lane != 0) return;
+    uint32_t stage = 0, phase = 0;
+    int pending = -1;   // stage whose bulk store may still be reading shared memory
+    bool ok = true;
+    for (uint32_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+      const uint32_t first = item_first[item];
+      if (item_first[item + 1] - first != 1) continue;
+      const Seg s = segs[first];
+      BulkPlan p;
+      if (!plan_bulk<TO_TENSORS>(s, flat, p)) continue;
+      for (uint32_t t = 0; t < p.ntiles; ++t) {
+        if (!mbar_wait(&sh.full[stage], phase, abort_flag)) {
+          raise_timeout(status, &sh);
+          ok = false;
+          break;
+        }
+        if (p.straight) {
+          uint32_t cnt = p.nfull - t * p.V;
+          if (cnt > p.V) cnt = p.V;
+          bulk_s2g(p.dst + (size_t)t * p.V * 16u, ring + (size_t)stage * kStageBytes, cnt * 16u);
+          bulk_commit();
+          if (pending >= 0) {
+            bulk_wait_read<1>();
+            mbar_arrive(&sh.empty[pending]);
+          }
+          pending = (int)stage;
+        } else {
+          if (pending >= 0) {
+            bulk_wait_read<0>();
+            mbar_arrive(&sh.empty[pending]);
+            pending = -1;
+          }
+          mbar_arrive(&sh.empty[stage]);   // the consumers write this stage's data themselves
+        }
+        if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    bulk_wait_read<0>();
+    if (pending >= 0) mbar_arrive(&sh.empty[pending]);
+    bulk_wait_all();
+    return;
+  }
+
+  // ---------------- consumers
+  const uint32_t c = threadIdx.x;   // 0 .. kConsThreads-1
+  Cksum ck;
+  u64 total = 0;
+  uint32_t cur = 0xffffffffu;
+  uint32_t stage = 0, phase = 0;
+  bool ok = true;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t first = item_first[item], last = item_first[item + 1];
+    if (PACK) {
+      const uint32_t bucket = segs[first].bucket;
+      if (bucket != cur) {   // uniform over the consumers
+        if (cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur, &sh);
+        total = 0;
+        cur = bucket;
+      }
+    }
+    const bool single = (last - first == 1);
+    BulkPlan p;
+    Seg s0;
+    bool bulk = false;
+    if (single) {
+      s0 = segs[first];
+      bulk = plan_bulk<TO_TENSORS>(s0, flat, p);
+    }
+    if (!bulk) {
+      if (!ok) continue;
+      const uint32_t g = single ? c : lane, G = single ? (uint32_t)kConsThreads : 32u;
+      for (uint32_t i = first + (single ? 0u : warp); i < last; i += (single ? 1u : (uint32_t)kConsWarps)) {
+        const Seg s = segs[i];
+        if (PACK) {
+          pack_piece(s, flat, g, G, ck);
+          total += ck.finish(s.word0);
+        } else {
+          uint8_t* t = reinterpret_cast<uint8_t*>(s.tensor);
+          uint8_t* f = flat + s.off;
+          copy_piece(TO_TENSORS ? t : f, TO_TENSORS ? f : t, s.nbytes, g, G);
+        }
+      }
+      continue;
+    }
+    // After a timeout the consumers keep walking the item list without touching memory, so that
+    // every consumer still meets the others at the checksum barriers.
+    if (!ok) continue;
+    // bulk piece: head bytes directly, full vectors through the ring, tail (and padding) directly
+    if (2 * c < p.head) st2(p.dst - p.head + 2 * c, ld2(p.src - p.head + 2 * c));
+    const uint32_t ws = p.a >> 2, bs = (p.a & 3) * 8;
+    for (uint32_t t = 0; t < p.ntiles; ++t) {
+      if (!mbar_wait(&sh.full[stage], phase, abort_flag)) {
+        raise_timeout(status, &sh);
+        ok = false;
+        break;
+      }
+      uint32_t cnt = p.nfull - t * p.V;
+      if (cnt > p.V) cnt = p.V;
+      const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageBytes);
+      const uint32_t vbase = t * p.V;
+      uint8_t* d = p.dst + (size_t)vbase * 16u;
+      if (p.straight) {
+        if (PACK) {   // the store thread moves the data; only the checksum is left to do
+#pragma unroll 4
+          for (uint32_t v = c; v < cnt; v += kConsThreads) ck.add(sp[v], vbase + v);
+        }
+      } else {
+#pragma unroll 2
+        for (uint32_t v = c; v < cnt; v += kConsThreads) {
+          const uint4 x = shift_pair(sp[v], sp[v + 1], ws, bs);
+          st16(d + (size_t)v * 16u, x);
+          if (PACK) ck.add(x, vbase + v);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.empty[stage]);
+      if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
+    }
+    if (!ok) continue;
+    if (PACK) {
+      // the vector with the tensor's last (n mod 16) bytes, then whole vectors of zero padding
+      const uint32_t nvec = (s0.nbytes + s0.pad) >> 4;
+      for (uint32_t v = p.nfull + c; v < nvec; v += kConsThreads) {
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        if (v == p.nfull && p.rem != 0) {
+          const uint8_t* tl = p.src + (size_t)p.nfull * 16u;
+#pragma unroll
+          for (uint32_t h = 0; h < 7; ++h)
+            if (2 * h < p.rem) w[h >> 1] |= ld2(tl + 2 * h) << ((h & 1) * 16);
+        }
+        const uint4 x = make_uint4(w[0], w[1], w[2], w[3]);
+        st16(p.dst + (size_t)v * 16u, x);
+        ck.add(x, v);
+      }
+      total += ck.finish(s0.word0);
+    } else {
+      const size_t tl = (size_t)p.nfull * 16u;
+      const uint32_t gt = kConsThreads - 1 - c;
+      if (2 * gt < p.rem) st2(p.dst + tl + 2 * gt, ld2(p.src + tl + 2 * gt));
+    }
+  }
+  if (PACK && cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur, &sh);
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+
+template <typename K>
+static int launch_ring(K kernel, const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
+                       unsigned long long* d_checksums, int* d_status, void* stream) {
+  int sms = 0;
+  int rc = device_sm_count(&sms);
+  if (rc != 0) return rc;
+  const size_t smem = (size_t)kRingStages * kStageBytes;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return (int)e;
+  uint64_t grid = (uint64_t)sms * tuning().ring_ctas_per_sm;
+  if (grid > n_items) grid = n_items;
+  if (grid == 0) grid = 1;
+  kernel<<<(uint32_t)grid, kRingThreads, smem, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat,
+                                                                    d_checksums, d_status);
+  count_launch();
+  return (int)cudaGetLastError();
+}
+
+int launch_pack_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
+                     unsigned long long* d_checksums, int* d_status, void* stream) {
+  return launch_ring(ring_kernel<true, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
+                     stream);
+}
+
+int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
+                     bool to_tensors, int* d_status, void* stream) {
+  if (to_tensors)
+    return launch_ring(ring_kernel<false, true>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
+  return launch_ring(ring_kernel<false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
+}
+
+}  // namespace tms

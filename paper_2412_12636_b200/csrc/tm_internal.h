@@ -51,7 +51,9 @@ struct Tuning {
   uint64_t small_bytes;    // pieces below this share items
   uint64_t group_bytes;    // byte budget of a shared item
   uint32_t group_max;      // piece budget of a shared item
-  uint32_t ctas_per_sm;    // persistent grid = SMs * ctas_per_sm
+  uint32_t ctas_per_sm;    // persistent grid = SMs * ctas_per_sm (register-path kernels)
+  uint32_t ring_ctas_per_sm;  // same for the bulk-copy ring kernels (96 KiB of shared memory each)
+  bool use_ring;           // pack / unpack / shard through the bulk-copy ring kernels
 };
 const Tuning& tuning();
 
@@ -72,6 +74,11 @@ int launch_pack(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_item
 // flat -> tensors when to_tensors, tensors -> flat otherwise (no checksum, no padding)
 int launch_copy(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
                 bool to_tensors, int* d_status, void* stream);
+// bulk-copy ring versions (ring_kernels.cu); d_status receives TM_ERR_TIMEOUT if a bounded wait expires
+int launch_pack_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
+                     unsigned long long* d_checksums, int* d_status, void* stream);
+int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
+                     bool to_tensors, int* d_status, void* stream);
 int launch_checksum(const uint8_t* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
                     unsigned long long* d_checksums, void* stream);
 int device_sm_count(int* sms);

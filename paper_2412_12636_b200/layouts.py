@@ -184,6 +184,11 @@ class RoleState:
         """(address, nbytes, elem_size, plane) per tensor."""
         return [(t.data_ptr(), s.nbytes, s.elem_size, s.plane) for s, t in zip(self.specs, self.tensors)]
 
+    def descs_of(self, indices: Sequence[int]) -> List[Tuple[int, int, int, int]]:
+        """Descriptors of a subset of the tensors, in the order given."""
+        return [(self.tensors[i].data_ptr(), self.specs[i].nbytes, self.specs[i].elem_size, self.specs[i].plane)
+                for i in indices]
+
     def plane_indices(self, plane: int) -> List[int]:
         return [i for i, s in enumerate(self.specs) if s.plane == plane]
 

@@ -31,7 +31,7 @@ def main() -> None:
     buckets, fused, alone = mover.alloc_buckets(), mover.alloc_checksums(), mover.alloc_checksums()
     shards = []
     for plane in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V):
-        ex = ShardExtractor([target.descs()[i] for i in target.plane_indices(plane)], cfg.shard_r, cfg.shard_D)
+        ex = ShardExtractor(target.descs_of(target.plane_indices(plane)), cfg.shard_r, cfg.shard_D)
         shards.append((ex, ex.alloc_out()))
     for _ in range(args.reps):
         mover.pack(buckets, fused)

@@ -84,7 +84,7 @@ def check_pack_against_oracle(oracle, state: layouts.RoleState, bucket_bytes: Op
 def check_shard_against_oracle(oracle, state: layouts.RoleState, indices: Sequence[int], r: int, D: int,
                                out_misalign: int = 0):
     """One shard of the plane made of tensors `indices` (common element size), vs the oracle."""
-    descs = [state.descs()[i] for i in indices]
+    descs = state.descs_of(indices)
     e = descs[0][2]
     host = [state.host_bytes(i) for i in indices]
     expect = oracle.shard(host, [h.size for h in host], e, r, D)

@@ -72,7 +72,7 @@ def check_unpack_on_device(state, buckets, B):
 
 def check_shard_sampled(oracle, state, indices, r, D):
     """Shard r of D of the plane `indices`: oracle gets host copies of only the tensors it crosses."""
-    descs = [state.descs()[i] for i in indices]
+    descs = state.descs_of(indices)
     e = descs[0][2]
     counts = [d[1] // e for d in descs]
     N = sum(counts)
@@ -147,7 +147,7 @@ def test_adversarial_20000_tensors_single_launch(oracle_mod):
     del buckets
     # shard extract for every r of 64 over the fp32 subset: exact union coverage, oracle on samples
     idx = state.elem_size_indices(4)
-    descs = [state.descs()[i] for i in idx]
+    descs = state.descs_of(idx)
     flat = torch.cat([state.tensors[i] for i in idx])
     parts = []
     for r in range(64):
@@ -213,7 +213,7 @@ def test_adversarial_200000_tensors_in_waves(oracle_mod):
         del buckets, alone
         idx = state.elem_size_indices(4)
         if idx:
-            descs = [state.descs()[i] for i in idx]
+            descs = state.descs_of(idx)
             flat = torch.cat([state.tensors[i] for i in idx])
             parts = []
             for r in range(64):

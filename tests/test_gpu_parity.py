@@ -83,7 +83,7 @@ def test_small_adversarial_full(oracle_mod):
         flat = np.concatenate([state.host_bytes(i) for i in idx])
         parts = []
         for r in range(0, 64):
-            ex = ShardExtractor([state.descs()[i] for i in idx], r, 64)
+            ex = ShardExtractor(state.descs_of(idx), r, 64)
             out = ex.alloc_out()
             ex.extract(out)
             parts.append(out.cpu().numpy())
