@@ -35,6 +35,10 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 WORKLOADS = {"cfg0": 0, "cfg1": 1, "cfg2": 2, "cfg3": 3}
+# DRAM bytes (read + written) per algorithmic byte of the pack kernel, from the ncu capture summarised
+# in profiles/; None until the current kernel has been captured.
+RING_PACK_TRAFFIC_PER_ALGORITHMIC_BYTE = None
+TRAFFIC_NOTE = "no ncu capture of the current kernel yet"
 
 
 # ------------------------------------------------------------------------------------------------
@@ -255,9 +259,90 @@ def run_reference(args) -> None:
 # the CUDA path
 
 
+class RoleBench:
+    """One role on the current GPU with every buffer the step needs."""
+
+    def __init__(self, workload: str):
+        from paper_2412_12636_b200 import layouts
+        from paper_2412_12636_b200.mover import RoleMover, ShardExtractor
+        if workload == "cfg4lite":
+            self.state = layouts.materialize_adversarial(layouts.adversarial_specs(20_000), "cuda")
+            self.name, self.bucket_bytes, self.shard_r, self.shard_D = "adversarial-20000", layouts.ADVERSARIAL_BUCKET, 29, 64
+            planes = [self.state.elem_size_indices(4)]
+        else:
+            cfg = layouts.role_config(WORKLOADS[workload])
+            self.state = layouts.materialize(cfg, "cuda")
+            self.name, self.bucket_bytes, self.shard_r, self.shard_D = cfg.name, cfg.bucket_bytes, cfg.shard_r, cfg.shard_D
+            planes = [self.state.plane_indices(p) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)]
+        state = self.state
+        self.target = layouts.blank_like(state)
+        self.mover = RoleMover(state.descs(), self.bucket_bytes)
+        self.unmover = RoleMover(self.target.descs(), self.bucket_bytes)
+        self.buckets = self.mover.alloc_buckets()
+        self.cks_fused = self.mover.alloc_checksums()
+        self.cks_alone = self.mover.alloc_checksums()
+        self.shards = []
+        for idx in planes:
+            ex = ShardExtractor(self.target.descs_of(idx), self.shard_r, self.shard_D)
+            self.shards.append((ex, ex.alloc_out()))
+        self.per_op = step_bytes(state.state_bytes, self.mover.total_bytes, self.mover.n_buckets,
+                                 [ex.out_bytes for ex, _ in self.shards])
+        self.bytes_per_step = sum(self.per_op.values())
+        self.stream = torch.cuda.current_stream()
+
+    def one_step(self, events=None):
+        marks = []
+
+        def mark():
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(self.stream)
+                marks.append(e)
+        mark()
+        self.mover.pack(self.buckets, self.cks_fused)
+        mark()
+        self.mover.checksum(self.buckets, self.cks_alone)
+        mark()
+        self.unmover.unpack(self.buckets)
+        mark()
+        for ex, out in self.shards:
+            ex.extract(out)
+        mark()
+        if events is not None:
+            events.append(marks)
+
+    def timed(self, steps: int):
+        """(elapsed ms over `steps` steps, mean ms per operation)."""
+        op_events: List[list] = []
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(self.stream)
+        for _ in range(steps):
+            self.one_step(op_events)
+        end.record(self.stream)
+        torch.cuda.synchronize()
+        names = ["pack", "checksum", "unpack", "shard"]
+        op_ms = {n: statistics.mean(m[i].elapsed_time(m[i + 1]) for m in op_events) for i, n in enumerate(names)}
+        return start.elapsed_time(end), op_ms
+
+    def self_check(self) -> bool:
+        from paper_2412_12636_b200 import layouts
+        ok = self.mover.status() == 0 and self.unmover.status() == 0
+        ok = ok and bool(torch.equal(self.cks_fused, self.cks_alone))
+        return ok and all(torch.equal(layouts.tensor_bytes(a), layouts.tensor_bytes(b))
+                          for a, b in zip(self.state.tensors[:8], self.target.tensors[:8]))
+
+    def ops_report(self, op_ms: Dict[str, float], peak: float) -> Dict[str, dict]:
+        def entry(nbytes, ms):
+            g = gbs(nbytes, ms)
+            return {"ms": round(ms, 4), "GB/s": round(g, 1), "frac_of_measured_copy": round(g / peak, 4),
+                    "frac_of_8TBs_nominal": round(g / NOMINAL_HBM_GBS, 4)}
+        ops = {n: entry(self.per_op[n], op_ms[n]) for n in ("pack", "checksum", "unpack", "shard")}
+        ops["pack+checksum+shard"] = entry(self.per_op["pack"] + self.per_op["shard"], op_ms["pack"] + op_ms["shard"])
+        return ops
+
+
 def run_ours(args) -> None:
-    from paper_2412_12636_b200 import binding, layouts
-    from paper_2412_12636_b200.mover import RoleMover, ShardExtractor
+    from paper_2412_12636_b200 import binding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -269,44 +354,9 @@ def run_ours(args) -> None:
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    cfg = layouts.role_config(WORKLOADS[args.workload])
-    state = layouts.materialize(cfg, "cuda")
-    target = layouts.blank_like(state)
-    mover = RoleMover(state.descs(), cfg.bucket_bytes)
-    unmover = RoleMover(target.descs(), cfg.bucket_bytes)
-    buckets = mover.alloc_buckets()
-    cks_fused = mover.alloc_checksums()
-    cks_alone = mover.alloc_checksums()
-    shards = []
-    for plane in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V):
-        ex = ShardExtractor(target.descs_of(target.plane_indices(plane)), cfg.shard_r, cfg.shard_D)
-        shards.append((ex, ex.alloc_out()))
-    per_op = step_bytes(state.state_bytes, mover.total_bytes, mover.n_buckets, [ex.out_bytes for ex, _ in shards])
-    bytes_per_step = sum(per_op.values())
-    stream = torch.cuda.current_stream()
-
-    def one_step(events=None):
-        marks = []
-        def mark():
-            if events is not None:
-                e = torch.cuda.Event(enable_timing=True)
-                e.record(stream)
-                marks.append(e)
-        mark()
-        mover.pack(buckets, cks_fused)
-        mark()
-        mover.checksum(buckets, cks_alone)
-        mark()
-        unmover.unpack(buckets)
-        mark()
-        for ex, out in shards:
-            ex.extract(out)
-        mark()
-        if events is not None:
-            events.append(marks)
-
+    role = RoleBench(args.workload)
     for _ in range(max(args.warmup, 3)):
-        one_step()
+        role.one_step()
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -316,51 +366,52 @@ def run_ours(args) -> None:
     if rank == 0:
         sampler.start()
     launches0 = binding.tm_launch_count()
-    op_events: List[list] = []
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record(stream)
-    for _ in range(args.steps):
-        one_step(op_events)
-    end.record(stream)
-    torch.cuda.synchronize()
-    elapsed_ms = start.elapsed_time(end)
+    elapsed_ms, op_ms = role.timed(args.steps)
     launches = binding.tm_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     if world > 1:
         dist.barrier()
         torch.cuda.synchronize()
-    assert mover.status() == 0 and unmover.status() == 0
-    ok = bool(torch.equal(cks_fused, cks_alone))
-    ok = ok and all(torch.equal(a, b) for a, b in zip(state.tensors[:8], target.tensors[:8]))
+    ok = role.self_check()
 
-    total_ms, total_bytes = aggregate_over_ranks(elapsed_ms, bytes_per_step * args.steps)
-
-    names = ["pack", "checksum", "unpack", "shard"]
-    op_ms = {n: statistics.mean(m[i].elapsed_time(m[i + 1]) for m in op_events) for i, n in enumerate(names)}
+    total_ms, total_bytes = aggregate_over_ranks(elapsed_ms, role.bytes_per_step * args.steps)
     peak, peak_kind = measured_hbm_peak()
-    ops = {n: {"ms": round(op_ms[n], 4), "GB/s": round(gbs(per_op[n], op_ms[n]), 1),
-               "frac_of_measured_copy": round(gbs(per_op[n], op_ms[n]) / peak, 4),
-               "frac_of_8TBs_nominal": round(gbs(per_op[n], op_ms[n]) / NOMINAL_HBM_GBS, 4)} for n in names}
-    pcs_bytes = per_op["pack"] + per_op["shard"]
-    pcs_ms = op_ms["pack"] + op_ms["shard"]
-    ops["pack+checksum+shard"] = {"ms": round(pcs_ms, 4), "GB/s": round(gbs(pcs_bytes, pcs_ms), 1),
-                                  "frac_of_measured_copy": round(gbs(pcs_bytes, pcs_ms) / peak, 4),
-                                  "frac_of_8TBs_nominal": round(gbs(pcs_bytes, pcs_ms) / NOMINAL_HBM_GBS, 4)}
-    achieved = gbs(per_op["pack"], op_ms["pack"])
-    roofline = {"bound": "hbm", "kernel": "pack_kernel (fused pack + checksum)", "achieved": round(achieved, 1),
+    ops = role.ops_report(op_ms, peak)
+    achieved = gbs(role.per_op["pack"], op_ms["pack"])
+    roofline = {"bound": "hbm", "kernel": "ring_kernel<pack> (fused pack + checksum)", "achieved": round(achieved, 1),
                 "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(achieved / peak, 4),
-                "traffic": None, "algorithmic_bytes_per_launch": per_op["pack"]}
+                "traffic": RING_PACK_TRAFFIC_PER_ALGORITHMIC_BYTE and int(RING_PACK_TRAFFIC_PER_ALGORITHMIC_BYTE * role.per_op["pack"]),
+                "traffic_note": TRAFFIC_NOTE, "algorithmic_bytes_per_launch": role.per_op["pack"]}
 
     e2e = None
     cpu_baseline = None
+    also = {}
     if rank == 0 and world == 1:
         if not args.no_e2e:
-            e2e = run_e2e(args, cfg, state, mover, buckets, cks_fused, bytes_per_step, one_step, shards)
-        if not args.no_cpu_baseline:
-            step, sample = oracle_sample_step(cfg)
+            e2e = run_e2e(args, role)
+        if not args.no_cpu_baseline and args.workload in WORKLOADS:
+            from paper_2412_12636_b200 import layouts
+            step, sample = oracle_sample_step(layouts.role_config(WORKLOADS[args.workload]))
             dt, nb = step()
             cpu_baseline = {"value": round(gbs(nb, dt * 1e3), 4), "unit": UNIT, "cores": 1, "kind": "oracle",
                             "sample": sample, "seconds": round(dt, 2), "host_cores_available": os.cpu_count()}
+    state_bytes, n_buckets, n_tensors = role.state.state_bytes, role.mover.n_buckets, len(role.state.specs)
+    name, bucket_bytes, shard = role.name, role.bucket_bytes, f"r={role.shard_r} of D={role.shard_D}"
+    bytes_per_step = role.bytes_per_step
+    if rank == 0 and world == 1 and args.also:
+        del role
+        torch.cuda.empty_cache()
+        for w in args.also.split(","):
+            other = RoleBench(w)
+            for _ in range(3):
+                other.one_step()
+            torch.cuda.synchronize()
+            ms, oms = other.timed(max(3, args.steps // 2))
+            also[f"{w}:{other.name}"] = {"GB/s": round(gbs(other.bytes_per_step * max(3, args.steps // 2), ms), 2),
+                                         "ops": other.ops_report(oms, peak), "self_check": "ok" if other.self_check() else "MISMATCH"}
+            ok = ok and also[f"{w}:{other.name}"]["self_check"] == "ok"
+            del other
+            torch.cuda.empty_cache()
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -370,23 +421,26 @@ def run_ours(args) -> None:
         "metric": METRIC, "value": round(gbs(total_bytes, total_ms), 2), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 4),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8/u64", "data": "synthetic",
-        "config": {"workload": f"{args.workload}:{cfg.name}", "state_bytes": state.state_bytes,
-                   "bucket_bytes": cfg.bucket_bytes, "n_buckets": mover.n_buckets, "n_tensors": len(state.specs),
-                   "shard": f"r={cfg.shard_r} of D={cfg.shard_D}, three fp32 planes", "parallelism": "replicas only",
+        "config": {"workload": f"{args.workload}:{name}", "state_bytes": state_bytes,
+                   "bucket_bytes": bucket_bytes, "n_buckets": n_buckets, "n_tensors": n_tensors,
+                   "shard": f"{shard}, fp32 planes", "parallelism": "replicas only",
                    "l2": "inputs (GBs) far larger than the 126 MB L2; no flush needed",
                    "step": "pack+fused checksum, stand-alone checksum, unpack, shard extract x3"},
         "bytes_per_step": bytes_per_step, "ops": ops, "roofline": roofline, "cpu_baseline": cpu_baseline,
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "self_check": "ok" if ok else "MISMATCH",
         "frac_of_8TBs_nominal": round(gbs(total_bytes, total_ms) / NOMINAL_HBM_GBS / world, 4),
+        "also": also,
     }
     print(json.dumps(line), flush=True)
     if not ok:
         raise SystemExit("self-check failed: fused and stand-alone checksums differ or round trip broke")
 
 
-def run_e2e(args, cfg, state, mover, buckets, cks, bytes_per_step, one_step, shards):
+def run_e2e(args, role):
     """Same step, but the role's tensors start in pinned host memory and the results (packed stream,
     checksums, shards) end in pinned host memory; the copies are inside the timed region."""
+    from paper_2412_12636_b200 import layouts
+    state, mover, buckets, cks, shards = role.state, role.mover, role.buckets, role.cks_fused, role.shards
     try:
         import psutil
         avail = psutil.virtual_memory().available
@@ -397,7 +451,6 @@ def run_e2e(args, cfg, state, mover, buckets, cks, bytes_per_step, one_step, sha
     if avail < 2 * (h2d + d2h) + (8 << 30):
         return {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "skipped": f"host has {avail >> 30} GiB available, pinned staging needs {(h2d + d2h) >> 30} GiB"}
-    from paper_2412_12636_b200 import layouts
     host_in = torch.empty(h2d, dtype=torch.uint8, pin_memory=True)
     host_out = torch.empty(d2h, dtype=torch.uint8, pin_memory=True)
     views, pos = [], 0
@@ -413,7 +466,7 @@ def run_e2e(args, cfg, state, mover, buckets, cks, bytes_per_step, one_step, sha
     def e2e_step():
         for t, v in zip(state.tensors, views):
             layouts.tensor_bytes(t).copy_(v, non_blocking=True)
-        one_step()
+        role.one_step()
         o = 0
         host_out[o:o + mover.total_bytes].copy_(buckets, non_blocking=True)
         o += mover.total_bytes
@@ -435,7 +488,7 @@ def run_e2e(args, cfg, state, mover, buckets, cks, bytes_per_step, one_step, sha
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - t0) * 1e3 / k
     ms = s.elapsed_time(e) / k
-    return {"value": round(gbs(bytes_per_step, max(ms, wall_ms)), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": round(gbs(role.bytes_per_step, max(ms, wall_ms)), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": round(max(ms, wall_ms), 3), "steps": k,
             "note": "role tensors start and results end in pinned host memory; PCIe-bound"}
 
@@ -446,7 +499,8 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg3")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS) + ["cfg4lite"], default="cfg3")
+    ap.add_argument("--also", default="cfg2", help="comma-separated further workloads measured after the main one (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler launch lists)")
     args = ap.parse_args()
