@@ -37,8 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 WORKLOADS = {"cfg0": 0, "cfg1": 1, "cfg2": 2, "cfg3": 3}
 # DRAM bytes (read + written) per algorithmic byte of the pack kernel, from the ncu capture summarised
 # in profiles/; None until the current kernel has been captured.
-RING_PACK_TRAFFIC_PER_ALGORITHMIC_BYTE = None
-TRAFFIC_NOTE = "no ncu capture of the current kernel yet"
+RING_PACK_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.983
+TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum of ring_kernel<pack> captured on config 3 reduced to one "
+                "layer (2.944896 GB for 2.995192 GB algorithmic), scaled by bytes moved; "
+                "profiles/ring_kernel_pack_unpack_cfg3_1layer_ncu_full.md")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -438,8 +440,12 @@ def run_ours(args) -> None:
 
 def run_e2e(args, role):
     """Same step, but the role's tensors start in pinned host memory and the results (packed stream,
-    checksums, shards) end in pinned host memory; the copies are inside the timed region."""
+    checksums, shards) end in pinned host memory; every copy is inside the timed region.  The role is
+    cut into waves of whole buckets so that the three legs overlap: host->device copies of wave i+1
+    (copy stream), pack of wave i (compute stream), device->host copy of wave i-1's buckets (second
+    copy stream).  The stand-alone checksum, unpack and shard extract follow on the compute stream."""
     from paper_2412_12636_b200 import layouts
+    from paper_2412_12636_b200.mover import WaveMover
     state, mover, buckets, cks, shards = role.state, role.mover, role.buckets, role.cks_fused, role.shards
     try:
         import psutil
@@ -461,36 +467,65 @@ def run_e2e(args, role):
         views.append(v)
         pos += n
     torch.cuda.synchronize()
-    stream = torch.cuda.current_stream()
+    compute = torch.cuda.current_stream()
+    up, down = torch.cuda.Stream(), torch.cuda.Stream()
+    wave_bytes = max(role.bucket_bytes, 1 << 30)
+    wm = WaveMover(state.descs(), role.bucket_bytes, wave_bytes)
+    torch.cuda.synchronize()
+    dev_bytes = [layouts.tensor_bytes(t) for t in state.tensors]
 
     def e2e_step():
-        for t, v in zip(state.tensors, views):
-            layouts.tensor_bytes(t).copy_(v, non_blocking=True)
-        role.one_step()
-        o = 0
-        host_out[o:o + mover.total_bytes].copy_(buckets, non_blocking=True)
-        o += mover.total_bytes
+        copied = 0   # tensors [0, copied) have their host->device copy enqueued
+        up.wait_stream(compute)     # the previous step's readers of the tensors are done
+        down.wait_stream(compute)
+        for i, w in enumerate(wm.waves):
+            first, last = wm.tensor_ranges[i]
+            with torch.cuda.stream(up):
+                for k in range(copied, last):
+                    dev_bytes[k].copy_(views[k], non_blocking=True)
+                copied = max(copied, last)
+                arrived = torch.cuda.Event()
+                arrived.record(up)
+            compute.wait_event(arrived)
+            wm.pack_wave(i, buckets, cks, compute)
+            packed = torch.cuda.Event()
+            packed.record(compute)
+            with torch.cuda.stream(down):
+                down.wait_event(packed)
+                host_out[w.stream_begin:w.stream_end].copy_(buckets[w.stream_begin:w.stream_end], non_blocking=True)
+        role.mover.checksum(buckets, role.cks_alone)
+        role.unmover.unpack(buckets)
+        for ex, out in shards:
+            ex.extract(out)
+        o = mover.total_bytes
         host_out[o:o + 8 * mover.n_buckets].copy_(cks.view(torch.uint8), non_blocking=True)
         o += 8 * mover.n_buckets
         for ex, out in shards:
             host_out[o:o + ex.out_bytes].copy_(out, non_blocking=True)
             o += ex.out_bytes
+        compute.wait_stream(down)
 
     e2e_step()
     torch.cuda.synchronize()
+    T = mover.total_bytes
+    ok = role.self_check()
+    for lo in (0, (T // 2) & ~255, max(0, T - (1 << 20))):
+        hi = min(T, lo + (1 << 20))
+        ok = ok and bool(torch.equal(host_out[lo:hi], buckets[lo:hi].cpu()))
     k = max(1, min(args.steps, 3))
     t0 = time.perf_counter()
     s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s.record(stream)
+    s.record(compute)
     for _ in range(k):
         e2e_step()
-    e.record(stream)
+    e.record(compute)
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - t0) * 1e3 / k
     ms = s.elapsed_time(e) / k
     return {"value": round(gbs(role.bytes_per_step, max(ms, wall_ms)), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": round(max(ms, wall_ms), 3), "steps": k,
-            "note": "role tensors start and results end in pinned host memory; PCIe-bound"}
+            "waves": len(wm.waves), "self_check": "ok" if ok else "MISMATCH",
+            "note": "role tensors start and results end in pinned host memory; copies overlap the pack wave by wave; PCIe-bound"}
 
 
 def main() -> None:

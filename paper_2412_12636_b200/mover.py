@@ -72,3 +72,37 @@ class ShardExtractor:
         return binding.tm_shard_extract(self.descs, self.r, self.D, out.data_ptr(),
                                         out.numel() * out.element_size(), self.workspace.data_ptr(),
                                         self.workspace.numel(), _stream_handle(stream))
+
+
+class WaveMover:
+    """The same role cut into waves of whole buckets (see waves.py), one plan per wave.
+
+    Wave i packs into stream bytes [begin_i, end_i) and produces the checksums of its own buckets,
+    so waves can be packed one after another — into slices of one full-size buffer, or into a
+    small ring of staging slots when the packed copy must not take a second role's worth of memory
+    (the paper's §8.5 rule: the transfer channel is a bounded, recycled buffer).  The concatenation
+    of the waves' streams and checksum lists equals what a single plan produces."""
+
+    def __init__(self, descs: Sequence[Tuple[int, int, int, int]], bucket_bytes: int, wave_bytes: int,
+                 device="cuda", stream: Optional[torch.cuda.Stream] = None):
+        from . import waves as _waves
+        whole = binding.Plan(descs, bucket_bytes)
+        self.total_bytes, self.n_buckets, self.bucket_bytes = whole.total_bytes, whole.n_buckets, bucket_bytes
+        offsets = whole.offsets()
+        whole.close()
+        sizes = [d[1] for d in descs]
+        self.waves = _waves.cut_waves(sizes, offsets, self.total_bytes, bucket_bytes, wave_bytes)
+        self.movers = []
+        self.tensor_ranges = []   # per wave: (first tensor, last tensor + 1) touched by the wave
+        for w in self.waves:
+            part_descs = [(descs[p.tensor][0] + p.byte_start, p.nbytes, descs[p.tensor][2], descs[p.tensor][3])
+                          for p in w.parts]
+            self.movers.append(RoleMover(part_descs, bucket_bytes, device, stream))
+            self.tensor_ranges.append((w.parts[0].tensor, w.parts[-1].tensor + 1))
+
+    def pack_wave(self, i: int, buckets: torch.Tensor, checksums: Optional[torch.Tensor],
+                  stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Packs wave i into its slice of the full-size `buckets` / `checksums` tensors."""
+        w = self.waves[i]
+        cks = None if checksums is None else checksums[w.first_bucket:w.first_bucket + w.n_buckets]
+        self.movers[i].pack(buckets[w.stream_begin:w.stream_end], cks, stream)

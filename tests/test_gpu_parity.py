@@ -171,3 +171,22 @@ def test_repeated_runs_are_identical():
     first = b1.clone()
     _, b2, c2 = G.gpu_pack(state, 1 << 18)
     assert torch.equal(first, b2) and np.array_equal(c1, c2)
+
+
+@pytest.mark.parametrize("wave_bytes", [1 << 20, 3 << 20, 1 << 30])
+def test_wave_by_wave_pack_equals_single_plan_and_oracle(oracle_mod, wave_bytes):
+    from paper_2412_12636_b200.mover import WaveMover
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    exp_stream, exp_cks = oracle_mod.pack(G.host_tensors(state), cfg.bucket_bytes)
+    wm = WaveMover(state.descs(), cfg.bucket_bytes, wave_bytes)
+    assert (wm.total_bytes, wm.n_buckets) == (exp_stream.size, exp_cks.size)
+    assert len(wm.waves) == -(-wm.n_buckets // max(1, wave_bytes // cfg.bucket_bytes))
+    whole, buckets = G.guarded(wm.total_bytes)
+    cks = torch.zeros(wm.n_buckets, dtype=torch.int64, device="cuda")
+    for i in reversed(range(len(wm.waves))):          # order does not matter: waves are independent
+        wm.pack_wave(i, buckets, cks)
+    torch.cuda.synchronize()
+    assert G.guards_intact(whole, wm.total_bytes)
+    assert np.array_equal(buckets.cpu().numpy(), exp_stream)
+    assert np.array_equal(G.u64(cks), exp_cks)
