@@ -50,8 +50,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_unpack.argtypes = [_p, _p, _u64, _p, _u64]
         L.oracle_shard_bounds.argtypes = [_u64, _u32, _u32, _p, _p]
         L.oracle_shard.argtypes = [_p, _p, _u64, _u32, _u32, _u32, _p, _u64, _p]
+        L.oracle_shard_insert.argtypes = [_p, _p, _u64, _u32, _u32, _u32, _p, _u64, _p]
         for name in ("oracle_layout", "oracle_checksum", "oracle_pack", "oracle_pack_range",
-                     "oracle_unpack", "oracle_shard_bounds", "oracle_shard"):
+                     "oracle_unpack", "oracle_shard_bounds", "oracle_shard", "oracle_shard_insert"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -160,3 +161,19 @@ def shard(tensors: Sequence[Optional[np.ndarray]], nbytes: Sequence[int], elem_s
                               out.ctypes.data if cap else None, cap, ctypes.addressof(got)),
            "shard")
     return out[: int(got.value) * elem_size]
+
+
+def shard_insert(tensors: Sequence[Optional[np.ndarray]], nbytes: Sequence[int], elem_size: int, r: int,
+                 D: int, data: np.ndarray) -> int:
+    """Writes `data` (shard r of D) into the plane's tensors IN PLACE (uint8 arrays); tensors the
+    shard does not touch may be None.  Returns the number of elements written."""
+    for t in tensors:
+        assert t is None or (t.dtype == np.uint8 and t.flags.c_contiguous and t.flags.writeable)
+    sz = _sizes(nbytes)
+    d = _as_bytes(data)
+    got = _u64(0)
+    ptrs = _ptr_table(tensors)
+    _check(lib().oracle_shard_insert(ptrs, sz.ctypes.data, len(tensors), elem_size, r, D,
+                                     d.ctypes.data if d.size else None, d.size, ctypes.addressof(got)),
+           "shard_insert")
+    return int(got.value)

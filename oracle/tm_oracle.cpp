@@ -215,4 +215,36 @@ int oracle_shard(const uint8_t* const* ptrs, const uint64_t* nbytes, uint64_t n,
   return ORC_OK;
 }
 
+// Inverse of oracle_shard: element g of the flat plane, for g in [lo, hi), is overwritten with
+// element g - lo of `in`; every other element of every tensor is left as it is.
+int oracle_shard_insert(uint8_t* const* ptrs, const uint64_t* nbytes, uint64_t n, uint32_t e,
+                        uint32_t r, uint32_t D, const uint8_t* in, uint64_t in_bytes,
+                        uint64_t* in_elems) {
+  if (ptrs == NULL || nbytes == NULL || n == 0) return ORC_ERR_ARG;
+  if (e != 2 && e != 4 && e != 8) return ORC_ERR_DTYPE;
+  uint64_t N = 0;
+  for (uint64_t k = 0; k < n; ++k) {
+    if (nbytes[k] == 0 || nbytes[k] % e != 0) return ORC_ERR_ARG;
+    N += nbytes[k] / e;
+  }
+  uint64_t lo = 0, hi = 0;
+  int rc = oracle_shard_bounds(N, r, D, &lo, &hi);
+  if (rc != ORC_OK) return rc;
+  if (in_elems != NULL) *in_elems = hi - lo;
+  if (hi == lo) return ORC_OK;
+  if (in == NULL) return ORC_ERR_ARG;
+  if (in_bytes < (hi - lo) * e) return ORC_ERR_CAPACITY;
+  uint64_t g = 0;
+  for (uint64_t k = 0; k < n; ++k) {
+    uint64_t count = nbytes[k] / e;
+    for (uint64_t idx = 0; idx < count; ++idx, ++g) {
+      if (g >= lo && g < hi) {
+        if (ptrs[k] == NULL) return ORC_ERR_ARG;
+        for (uint32_t b = 0; b < e; ++b) ptrs[k][idx * e + b] = in[(g - lo) * e + b];
+      }
+    }
+  }
+  return ORC_OK;
+}
+
 }  // extern "C"

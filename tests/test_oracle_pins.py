@@ -267,3 +267,40 @@ def test_shard_errors(oracle_mod):
     with pytest.raises(oracle_mod.OracleError) as ex:   # nbytes not a multiple of elem_size
         oracle_mod.shard([np.zeros(6, dtype=np.uint8)], [6], 4, 0, 1)
     assert ex.value.code == -1
+
+
+# ------------------------------------------------------------------ shard insert
+
+
+@pytest.mark.parametrize("e", [2, 4, 8])
+@pytest.mark.parametrize("D", [1, 3, 64])
+def test_shard_insert_brute_force_and_inverse(oracle_mod, e, D):
+    rng = np.random.default_rng(e * 1000 + D)
+    counts = [int(rng.choice([1, 3, 5, 127, 129, 257])) for _ in range(int(rng.integers(1, 7)))]
+    tensors = [rng.integers(0, 256, c * e, dtype=np.uint8) for c in counts]
+    sizes = [t.size for t in tensors]
+    flat = bytearray(b"".join(t.tobytes() for t in tensors))
+    N = len(flat) // e
+    for r in sorted({0, D // 2, D - 1}):
+        lo, hi = (r * N) // D, ((r + 1) * N) // D
+        data = rng.integers(0, 256, (hi - lo) * e, dtype=np.uint8)
+        work = [t.copy() for t in tensors]
+        assert oracle_mod.shard_insert(work, sizes, e, r, D, data) == hi - lo
+        expect = bytearray(flat)
+        expect[lo * e:hi * e] = data.tobytes()                         # Python slice assignment
+        assert b"".join(t.tobytes() for t in work) == bytes(expect)
+        assert oracle_mod.shard(work, sizes, e, r, D).tobytes() == data.tobytes()   # extract(insert(x)) == x
+    # inserting every shard of another plane rebuilds that plane
+    other = [rng.integers(0, 256, t.size, dtype=np.uint8) for t in tensors]
+    work = [t.copy() for t in tensors]
+    for r in range(D):
+        oracle_mod.shard_insert(work, sizes, e, r, D, oracle_mod.shard(other, sizes, e, r, D))
+    assert all(np.array_equal(a, b) for a, b in zip(work, other))
+
+
+def test_shard_insert_errors(oracle_mod):
+    t = [np.zeros(8, dtype=np.uint8)]
+    for e, r, D, n, code in ((4, 2, 2, 8, -5), (3, 0, 1, 8, -6), (4, 0, 1, 4, -3)):
+        with pytest.raises(oracle_mod.OracleError) as ex:
+            oracle_mod.shard_insert(t, [8], e, r, D, np.zeros(n, dtype=np.uint8))
+        assert ex.value.code == code
