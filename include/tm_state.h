@@ -156,6 +156,17 @@ int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, ui
                      void* d_out, uint64_t out_capacity, uint64_t* out_elems,
                      void* d_workspace, uint64_t workspace_bytes, void* stream);
 
+/* Shard insert: the inverse of tm_shard_extract (a joiner that fetched its slice of the optimizer
+ * state from a peer or from storage — §7 "State Synchronization", the no-redundancy case — puts it
+ * into its own flat plane).  Elements [lo, hi) of the plane (same definition and bounds as
+ * tm_shard_extract) are overwritten with the (hi - lo) elements at d_in (device, >= 2-byte aligned,
+ * `in_bytes` >= (hi-lo)*elem_size, no overlap with the tensors); all other elements stay as they
+ * are.  *in_elems (host, may be NULL) receives hi - lo.  Workspace: as for tm_shard_extract
+ * (tm_shard_workspace gives the size).  The tensors of the plane must not overlap one another. */
+int tm_shard_insert(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                    const void* d_in, uint64_t in_bytes, uint64_t* in_elems,
+                    void* d_workspace, uint64_t workspace_bytes, void* stream);
+
 /* Size of the library-resident scratch array used by tm_shard_extract_static. */
 #define TM_STATIC_SCRATCH_BYTES (1u << 20)
 

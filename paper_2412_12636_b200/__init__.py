@@ -8,7 +8,7 @@ attribute does, and fails loudly if it has not been built.
 """
 
 _BINDING_NAMES = (
-    "Plan", "TmError", "tm_state_pack", "tm_state_unpack", "tm_shard_extract", "tm_checksum",
+    "Plan", "TmError", "tm_state_pack", "tm_state_unpack", "tm_shard_extract", "tm_shard_insert", "tm_shard_extract_static", "tm_checksum",
     "tm_shard_bounds", "tm_shard_workspace", "tm_launch_count", "load_library", "make_descs",
 )
 

@@ -32,6 +32,7 @@ SIGNATURES = {
     "tm_shard_bounds": (_int, [_u64, _u32, _u32, _p, _p]),
     "tm_shard_workspace": (_int, [_p, _u64, _u32, _u32, _p]),
     "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
+    "tm_shard_insert": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
     "tm_shard_extract_static": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p]),
     "tm_workspace_status": (_int, [_p, _p, _p]),
     "tm_checksum": (_int, [_p, _u64, _u64, _p, _p]),
@@ -158,6 +159,16 @@ def tm_shard_extract(descs, r: int, D: int, d_out: int, out_capacity: int, d_wor
     n = _u64()
     _check(load_library().tm_shard_extract(arr, len(arr), r, D, d_out, out_capacity, ctypes.byref(n),
                                            d_workspace, workspace_bytes, stream), "tm_shard_extract")
+    return n.value
+
+
+def tm_shard_insert(descs, r: int, D: int, d_in: int, in_bytes: int, d_workspace: int, workspace_bytes: int,
+                    stream: int) -> int:
+    """Returns the number of elements written into the plane."""
+    arr = descs if isinstance(descs, ctypes.Array) else make_descs(descs)
+    n = _u64()
+    _check(load_library().tm_shard_insert(arr, len(arr), r, D, d_in, in_bytes, ctypes.byref(n), d_workspace,
+                                          workspace_bytes, stream), "tm_shard_insert")
     return n.value
 
 

@@ -167,9 +167,10 @@ int tm_shard_workspace(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, 
   return TM_OK;
 }
 
-int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, void* d_out,
-                     uint64_t out_capacity, uint64_t* out_elems, void* d_workspace,
-                     uint64_t workspace_bytes, void* stream) {
+// Shared body of shard extract (tensors -> flat) and shard insert (flat -> tensors).
+static int shard_run(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, void* d_flat,
+                     uint64_t flat_capacity, uint64_t* elems, void* d_workspace, uint64_t workspace_bytes,
+                     void* stream, bool to_tensors) {
   uint32_t e = 0;
   uint64_t n_elems = 0;
   int rc = tm_shard_validate(plane_descs, n_desc, r, D, &e, &n_elems);
@@ -177,18 +178,18 @@ int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, ui
   uint64_t lo = 0, hi = 0;
   rc = tm_bounds_u128(n_elems, r, D, &lo, &hi);
   if (rc != TM_OK) return rc;
-  if (out_elems != nullptr) *out_elems = hi - lo;
+  if (elems != nullptr) *elems = hi - lo;
   if (hi == lo) return TM_OK;
-  if (d_out == nullptr || d_workspace == nullptr) return TM_ERR_ARG;
-  if (((uintptr_t)d_out & 1) != 0 || ((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
-  const uint64_t out_bytes = (hi - lo) * e;
-  if (out_capacity < out_bytes) return TM_ERR_CAPACITY;
-  const uint64_t out_addr = (uint64_t)(uintptr_t)d_out;
+  if (d_flat == nullptr || d_workspace == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_flat & 1) != 0 || ((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+  const uint64_t flat_bytes = (hi - lo) * e;
+  if (flat_capacity < flat_bytes) return TM_ERR_CAPACITY;
+  const uint64_t flat_addr = (uint64_t)(uintptr_t)d_flat;
   for (uint64_t k = 0; k < n_desc; ++k)
-    if (ranges_overlap((uint64_t)(uintptr_t)plane_descs[k].ptr, plane_descs[k].nbytes, out_addr, out_bytes))
+    if (ranges_overlap((uint64_t)(uintptr_t)plane_descs[k].ptr, plane_descs[k].nbytes, flat_addr, flat_bytes))
       return TM_ERR_OVERLAP;
   tms::WorkList wl;
-  tm_shard_worklist(plane_descs, n_desc, e, lo, hi, out_addr, &wl);
+  tm_shard_worklist(plane_descs, n_desc, e, lo, hi, flat_addr, &wl);
   const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
   if (workspace_bytes < l.total) return TM_ERR_CAPACITY;
   rc = upload_worklist(wl, l, (uint8_t*)d_workspace, (cudaStream_t)stream);
@@ -196,9 +197,22 @@ int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, ui
   const uint8_t* ws = (const uint8_t*)d_workspace;
   auto copy_fn = tms::tuning().use_ring ? tms::launch_copy_ring : tms::launch_copy;
   int err = copy_fn((const tms::Seg*)(ws + l.segs_off), (const uint32_t*)(ws + l.items_off),
-                            (uint32_t)wl.n_items(), (uint8_t*)d_out, /*to_tensors=*/false,
-                            (int*)d_workspace, stream);
+                    (uint32_t)wl.n_items(), (uint8_t*)d_flat, to_tensors, (int*)d_workspace, stream);
   return err == 0 ? TM_OK : cuda_fail(err);
+}
+
+int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, void* d_out,
+                     uint64_t out_capacity, uint64_t* out_elems, void* d_workspace,
+                     uint64_t workspace_bytes, void* stream) {
+  return shard_run(plane_descs, n_desc, r, D, d_out, out_capacity, out_elems, d_workspace, workspace_bytes,
+                   stream, /*to_tensors=*/false);
+}
+
+int tm_shard_insert(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, const void* d_in,
+                    uint64_t in_bytes, uint64_t* in_elems, void* d_workspace, uint64_t workspace_bytes,
+                    void* stream) {
+  return shard_run(plane_descs, n_desc, r, D, const_cast<void*>(d_in), in_bytes, in_elems, d_workspace,
+                   workspace_bytes, stream, /*to_tensors=*/true);
 }
 
 int tm_workspace_status(const void* d_workspace, void* stream, int* device_status) {

@@ -189,6 +189,13 @@ class RoleState:
         return [(self.tensors[i].data_ptr(), self.specs[i].nbytes, self.specs[i].elem_size, self.specs[i].plane)
                 for i in indices]
 
+    def subset(self, indices: Sequence[int], name: Optional[str] = None) -> "RoleState":
+        """The same tensors restricted to `indices` (order kept) — e.g. the role delta between a middle
+        and a first/last pipeline stage: embedding / output layer and their optimizer state."""
+        return RoleState(name or f"{self.name}-subset", [self.specs[i] for i in indices],
+                         [self.tensors[i] for i in indices], self.bucket_bytes, self.shard_r, self.shard_D,
+                         self.arena)
+
     def plane_indices(self, plane: int) -> List[int]:
         return [i for i, s in enumerate(self.specs) if s.plane == plane]
 

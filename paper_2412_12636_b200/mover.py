@@ -73,6 +73,12 @@ class ShardExtractor:
                                         out.numel() * out.element_size(), self.workspace.data_ptr(),
                                         self.workspace.numel(), _stream_handle(stream))
 
+    def insert(self, data: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+        """Writes `data` (this shard) into the plane's tensors; the inverse of extract."""
+        return binding.tm_shard_insert(self.descs, self.r, self.D, data.data_ptr(),
+                                       data.numel() * data.element_size(), self.workspace.data_ptr(),
+                                       self.workspace.numel(), _stream_handle(stream))
+
 
 class WaveMover:
     """The same role cut into waves of whole buckets (see waves.py), one plan per wave.

@@ -190,3 +190,47 @@ def test_wave_by_wave_pack_equals_single_plan_and_oracle(oracle_mod, wave_bytes)
     assert G.guards_intact(whole, wm.total_bytes)
     assert np.array_equal(buckets.cpu().numpy(), exp_stream)
     assert np.array_equal(G.u64(cks), exp_cks)
+
+
+@pytest.mark.parametrize("e", [4, 2, 8])
+def test_shard_insert_matches_oracle_and_inverts_extract(oracle_mod, e):
+    specs = layouts.adversarial_specs(400, max_log2=17)
+    state = layouts.materialize_adversarial(specs, "cuda", seed=11)
+    idx = state.elem_size_indices(e)
+    descs = state.descs_of(idx)
+    sizes = [d[1] for d in descs]
+    before = state.arena.clone()
+    for r, D, mis in ((0, 1, 0), (3, 7, 2), (63, 64, 6), (5, 3 * sum(sizes), 0)):   # last: empty or 1-element shards
+        ex = ShardExtractor(descs, r, D)
+        gen = torch.Generator("cuda").manual_seed(r * 1000 + D)
+        whole = torch.randint(0, 256, (ex.out_bytes + 16,), dtype=torch.uint8, device="cuda", generator=gen)
+        data = whole[mis:mis + ex.out_bytes]
+        host = [state.host_bytes(i).copy() for i in idx]
+        assert oracle_mod.shard_insert(host, sizes, e, r, D, data.cpu().numpy()) == ex.hi - ex.lo
+        assert ex.insert(data) == ex.hi - ex.lo
+        torch.cuda.synchronize()
+        for i, h in zip(idx, host):
+            assert np.array_equal(state.host_bytes(i), h), f"tensor {i} after insert r={r} D={D}"
+        out = ex.alloc_out()
+        ex.extract(out)
+        torch.cuda.synchronize()
+        assert torch.equal(out, data)                       # extract(insert(x)) == x
+    # nothing outside the plane's tensors changed (gaps, tensors of other element sizes)
+    mask = torch.ones_like(before, dtype=torch.bool)
+    base = state.arena.data_ptr()
+    for i in idx:
+        o = state.tensors[i].data_ptr() - base
+        mask[o:o + state.specs[i].nbytes] = False
+    assert torch.equal(state.arena[mask], before[mask])
+
+
+def test_role_delta_pack_of_a_descriptor_subset(oracle_mod):
+    # A standby warmed as a middle stage that is promoted to a first/last stage only needs the extra
+    # layers' parameters and optimizer state (paper §6): pack just those descriptors.
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    delta = [i for i, s in enumerate(state.specs) if ".embedding" in s.name or ".final_ln" in s.name]
+    assert len(delta) == 12
+    sub = state.subset(delta, "tiny-gpt-first-stage-delta")
+    mover, _, stream = G.check_pack_against_oracle(oracle_mod, sub, 256 * 1024)
+    assert stream.size == sum(-(-s.nbytes // 256) * 256 for s in sub.specs)
