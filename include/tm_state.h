@@ -199,6 +199,14 @@ int tm_workspace_status(const void* d_workspace, void* stream, int* device_statu
 int tm_checksum(const void* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
                 uint64_t* d_checksums, void* stream);
 
+/* Self-test of the device-side failure reporting.  The kernels' only waits (mbarrier waits of the
+ * bulk-copy ring) are bounded in time; a wait that expires makes the kernel record TM_ERR_TIMEOUT in
+ * the status word of its workspace and return, leaving the context usable.  This call launches one
+ * thread that waits, for at most limit_ns (1 .. 5e9), on a barrier that nothing will ever complete,
+ * so that the reporting path can be checked without a fault or a hang: afterwards
+ * tm_workspace_status(d_workspace) yields TM_ERR_TIMEOUT.  d_workspace: >= 256 bytes, 256-byte aligned. */
+int tm_selftest_bounded_wait(void* d_workspace, uint64_t limit_ns, void* stream);
+
 /* ---- diagnostics ----------------------------------------------------------------------------- */
 
 const char* tm_strerror(int status);

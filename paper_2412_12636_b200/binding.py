@@ -34,6 +34,7 @@ SIGNATURES = {
     "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
     "tm_shard_insert": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
     "tm_shard_extract_static": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p]),
+    "tm_selftest_bounded_wait": (_int, [_p, _u64, _p]),
     "tm_workspace_status": (_int, [_p, _p, _p]),
     "tm_checksum": (_int, [_p, _u64, _u64, _p, _p]),
     "tm_strerror": (ctypes.c_char_p, [_int]),
@@ -180,6 +181,10 @@ def tm_shard_extract_static(descs, r: int, D: int, d_out: int, out_capacity: int
     _check(load_library().tm_shard_extract_static(arr, len(arr), r, D, d_out, out_capacity, ctypes.byref(n),
                                                   stream), "tm_shard_extract_static")
     return n.value
+
+
+def tm_selftest_bounded_wait(d_workspace: int, limit_ns: int, stream: int) -> None:
+    _check(load_library().tm_selftest_bounded_wait(d_workspace, limit_ns, stream), "tm_selftest_bounded_wait")
 
 
 def tm_workspace_status(d_workspace: int, stream: int) -> int:

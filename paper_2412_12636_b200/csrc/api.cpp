@@ -215,6 +215,14 @@ int tm_shard_insert(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uin
                    workspace_bytes, stream, /*to_tensors=*/true);
 }
 
+int tm_selftest_bounded_wait(void* d_workspace, uint64_t limit_ns, void* stream) {
+  if (d_workspace == nullptr || limit_ns == 0 || limit_ns > 5000000000ull) return TM_ERR_ARG;
+  if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+  TM_CUDA(cudaMemsetAsync(d_workspace, 0, tms::kStatusBlockBytes, (cudaStream_t)stream));
+  int e = tms::launch_wait_selftest((int*)d_workspace, limit_ns, stream);
+  return e == 0 ? TM_OK : cuda_fail(e);
+}
+
 int tm_workspace_status(const void* d_workspace, void* stream, int* device_status) {
   return read_status(d_workspace, (cudaStream_t)stream, device_status);
 }

@@ -60,7 +60,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 // Waits for the phase with the given parity; gives up after kWaitLimitNs or when the block aborts.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try(b, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
@@ -68,7 +69,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
     for (int i = 0; i < 64; ++i)
       if (mbar_try(b, parity)) return true;
     if (*abort_flag != 0) return false;
-    if (global_ns() - t0 > kWaitLimitNs) return false;
+    if (global_ns() - t0 > limit_ns) return false;
   }
 }
 // Non-multicast 1-D bulk copy global -> this block's shared memory, completion on an mbarrier.
@@ -365,7 +366,26 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
   if (PACK && cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur, &sh);
 }
 
+// Exercises the bounded wait on purpose: one thread waits for a barrier phase that nobody will ever
+// complete, gives up after limit_ns and reports TM_ERR_TIMEOUT through the status word, exactly as
+// the ring kernels do.  The kernel returns normally; nothing is left in flight.
+__global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ RingShared sh;
+  if (threadIdx.x == 0) {
+    mbar_init(&sh.full[0], 1);
+    sh.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(&sh.full[0], 0, &sh.abort_flag, limit_ns)) raise_timeout(status, &sh);
+  }
+}
+
 // ---- host side ------------------------------------------------------------------------------------
+
+int launch_wait_selftest(int* d_status, unsigned long long limit_ns, void* stream) {
+  wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d_status, limit_ns);
+  count_launch();
+  return (int)cudaGetLastError();
+}
 
 template <typename K>
 static int launch_ring(K kernel, const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,

@@ -239,3 +239,41 @@ def check_unpack_parts(state, buckets, B):
     torch.cuda.synchronize()
     assert um.status() == 0
     return targets
+
+
+def test_tensor_beyond_4_gib_and_word_index_beyond_2_31():
+    """Maximum sizes: one tensor of 2^31 + 4096 eight-byte words (16 GiB + 32 KiB) of a constant word.
+    Offsets exceed 32 bits, the tensor is cut into many pieces, and with a single 32 GiB bucket the
+    checksum weights 2i+1 exceed 2^32.  Closed form: n words of c give c * n^2 mod 2^64."""
+    M64 = 1 << 64
+    c = 0x0123456789ABCDEF
+    n = (1 << 31) + 4096
+    t = torch.full((n,), c, dtype=torch.int64, device="cuda")
+    spec = layouts.TensorSpec("big", n, torch.int64, layouts.PLANE_OTHER, 0)
+    state = layouts.RoleState("big", [spec], [t], 1 << 35, 0, 1)
+    for B in (1 << 35, 1 << 30):
+        mover = RoleMover(state.descs(), B)
+        assert mover.total_bytes == 8 * n and mover.n_buckets == -(-8 * n // B)
+        whole, buckets = G.guarded(mover.total_bytes)
+        cks, alone = mover.alloc_checksums(), mover.alloc_checksums()
+        mover.pack(buckets, cks)
+        mover.checksum(buckets, alone)
+        torch.cuda.synchronize()
+        assert mover.status() == 0 and G.guards_intact(whole, mover.total_bytes)
+        assert torch.equal(buckets.view(torch.int64), t)
+        words = [min(B // 8, n - j * (B // 8)) for j in range(mover.n_buckets)]
+        expect = [(c * w * w) % M64 for w in words]
+        assert [int(x) for x in G.u64(cks)] == expect
+        assert [int(x) for x in G.u64(alone)] == expect
+        back = torch.zeros_like(t)
+        um = RoleMover([(back.data_ptr(), 8 * n, 8, layouts.PLANE_OTHER)], B)
+        um.unpack(buckets)
+        torch.cuda.synchronize()
+        assert torch.equal(back, t)
+        del whole, buckets, back
+        torch.cuda.empty_cache()
+    ex = ShardExtractor(state.descs(), 2, 3)              # a 5.3 GiB slice starting beyond 4 GiB
+    out = ex.alloc_out()
+    assert ex.extract(out) == ex.hi - ex.lo
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int64), t[ex.lo:ex.hi])

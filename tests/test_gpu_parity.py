@@ -234,3 +234,22 @@ def test_role_delta_pack_of_a_descriptor_subset(oracle_mod):
     sub = state.subset(delta, "tiny-gpt-first-stage-delta")
     mover, _, stream = G.check_pack_against_oracle(oracle_mod, sub, 256 * 1024)
     assert stream.size == sum(-(-s.nbytes // 256) * 256 for s in sub.specs)
+
+
+def test_expired_device_wait_is_reported_not_hung():
+    # a wait that nothing completes: the kernel gives up after 50 ms, records the status and returns
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    assert binding.tm_workspace_status(ws.data_ptr(), s) == 0
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    binding.tm_selftest_bounded_wait(ws.data_ptr(), 50_000_000, s)
+    t1.record()
+    assert binding.tm_workspace_status(ws.data_ptr(), s) == binding.TM_ERR_TIMEOUT
+    assert 40.0 < t0.elapsed_time(t1) < 1000.0
+    # the context is still usable: a real operation right after
+    data = torch.ones(1 << 16, dtype=torch.int64, device="cuda")
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    binding.tm_checksum(data.data_ptr(), 8 << 16, 8 << 16, out.data_ptr(), s)
+    torch.cuda.synchronize()
+    assert int(G.u64(out)[0]) == (1 << 32)               # c * n^2 with c = 1, n = 2^16
