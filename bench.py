@@ -191,10 +191,10 @@ class ClockSampler:
 # CPU oracle timing (the cpu_baseline leg and --impl reference)
 
 
-def oracle_sample_step(cfg, device="cpu"):
-    """Builds the bounded sample — layer 0's tensors (for cfg0: the whole role) in all four planes —
-    on the host and returns a callable that runs the four oracle operations once over it,
-    returning (seconds, algorithmic bytes)."""
+def oracle_sample_step(cfg, n_layers=1):
+    """Builds the bounded sample — the tensors of the first `n_layers` layers (for cfg0: the whole
+    role) in all four planes — on the host and returns a callable that runs the four oracle
+    operations once over it, returning (seconds, algorithmic bytes)."""
     import numpy as np
     import oracle
     from paper_2412_12636_b200 import layouts
@@ -204,8 +204,9 @@ def oracle_sample_step(cfg, device="cpu"):
         keep = list(range(len(specs)))
         what = "whole role"
     else:
-        keep = [i for i, s in enumerate(specs) if ".l0." in s.name]
-        what = "layer 0 of every plane"
+        tags = tuple(f".l{i}." for i in range(n_layers))
+        keep = [i for i, s in enumerate(specs) if any(t in s.name for t in tags)]
+        what = f"layers 0..{n_layers - 1} of every plane"
     host = [layouts.tensor_bytes(layouts._fill_model_tensor(cfg, specs[i], torch.device("cpu"))).numpy() for i in keep]
     sizes = [h.size for h in host]
     fp32 = {p: [j for j, i in enumerate(keep) if specs[i].plane == p] for p in (1, 2, 3)}
@@ -235,13 +236,17 @@ def run_reference(args) -> None:
         return
     from paper_2412_12636_b200 import layouts
     cfg = layouts.role_config(WORKLOADS[args.workload])
-    step, sample = oracle_sample_step(cfg)
+    step, sample = oracle_sample_step(cfg, n_layers=1)
+    budget_s = 150.0                      # the whole run ends within a few minutes whatever --steps says
+    t_start = time.perf_counter()
     for _ in range(min(args.warmup, 1)):
         step()
     times, nbytes = [], 0
     for _ in range(max(1, args.steps)):
         dt, nbytes = step()
         times.append(dt)
+        if time.perf_counter() - t_start + dt > budget_s:
+            break
     ms = 1e3 * sum(times) / len(times)
     value = gbs(nbytes, ms)
     line = {
@@ -393,7 +398,7 @@ def run_ours(args) -> None:
             e2e = run_e2e(args, role)
         if not args.no_cpu_baseline and args.workload in WORKLOADS:
             from paper_2412_12636_b200 import layouts
-            step, sample = oracle_sample_step(layouts.role_config(WORKLOADS[args.workload]))
+            step, sample = oracle_sample_step(layouts.role_config(WORKLOADS[args.workload]), n_layers=4)
             dt, nb = step()
             cpu_baseline = {"value": round(gbs(nb, dt * 1e3), 4), "unit": UNIT, "cores": 1, "kind": "oracle",
                             "sample": sample, "seconds": round(dt, 2), "host_cores_available": os.cpu_count()}

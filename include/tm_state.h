@@ -42,7 +42,8 @@
  *   - The caller owns all device memory (tensors, packed buffer, checksum
  *     array, workspace) and the stream.  The library allocates no device
  *     memory.  A tm_plan owns host memory only, plus the contents it wrote
- *     into the workspace handed to tm_plan_upload.
+ *     into the workspace handed to tm_plan_upload.  The library keeps 8 MiB
+ *     of pinned host memory per GPU for uploading small work lists.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  All device work is enqueued on it and the call returns without
  *     waiting; the caller synchronises.  The device of the stream/pointers must

@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "tm_internal.h"
@@ -35,13 +36,84 @@ bool ranges_overlap(uint64_t a, uint64_t an, uint64_t b, uint64_t bn) {
   return a < b + bn && b < a + an;
 }
 
+// Pinned host staging for small work-list uploads: eight 1 MiB slots per device, reused round-robin;
+// a slot is free again once the copy that read it has completed (one event per slot).  Host memory
+// only.  With it an upload is one truly asynchronous copy instead of a memset plus two copies from
+// pageable memory that make the host wait for the stream.
+class HostStaging {
+ public:
+  static constexpr size_t kSlotBytes = 1u << 20;
+  static constexpr int kSlots = 8;
+  static constexpr int kMaxDevices = 64;
+
+  // Returns a slot for the current device (waiting for its previous copy), or -1 if unavailable.
+  int acquire(int dev) {
+    if (dev < 0 || dev >= kMaxDevices) return -1;
+    Pool& p = pools_[dev];
+    if (p.state == 0) {
+      p.state = -1;
+      uint8_t* base = nullptr;
+      if (cudaHostAlloc((void**)&base, kSlotBytes * kSlots, cudaHostAllocPortable) == cudaSuccess) {
+        bool ok = true;
+        for (int i = 0; i < kSlots && ok; ++i) {
+          p.host[i] = base + (size_t)i * kSlotBytes;
+          ok = cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming) == cudaSuccess;
+        }
+        if (ok) p.state = 1;
+      }
+      (void)cudaGetLastError();
+    }
+    if (p.state != 1) return -1;
+    const int i = p.next;
+    p.next = (p.next + 1) % kSlots;
+    if (p.busy[i] && cudaEventSynchronize(p.ev[i]) != cudaSuccess) return -1;
+    p.busy[i] = false;
+    return i;
+  }
+  uint8_t* host(int dev, int slot) { return pools_[dev].host[slot]; }
+  cudaError_t mark(int dev, int slot, cudaStream_t st) {
+    pools_[dev].busy[slot] = true;
+    return cudaEventRecord(pools_[dev].ev[slot], st);
+  }
+  std::mutex mutex;
+
+ private:
+  struct Pool {
+    int state = 0;   // 0 not tried, 1 ready, -1 unavailable
+    int next = 0;
+    uint8_t* host[kSlots] = {nullptr};
+    cudaEvent_t ev[kSlots] = {nullptr};
+    bool busy[kSlots] = {false};
+  };
+  Pool pools_[kMaxDevices];
+};
+HostStaging g_staging;
+
 int upload_worklist(const tms::WorkList& wl, const tms::WorkspaceLayout& l, uint8_t* d_ws, cudaStream_t st) {
+  const size_t items_bytes = wl.item_first.size() * sizeof(uint32_t);
+  const size_t segs_bytes = wl.segs.size() * sizeof(tms::Seg);
+  const size_t span = l.items_off + items_bytes;   // status block, pieces, items: one contiguous image
+  if (span <= HostStaging::kSlotBytes) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+      std::lock_guard<std::mutex> lock(g_staging.mutex);
+      const int slot = g_staging.acquire(dev);
+      if (slot >= 0) {
+        uint8_t* h = g_staging.host(dev, slot);
+        std::memset(h, 0, l.segs_off);
+        if (segs_bytes != 0) std::memcpy(h + l.segs_off, wl.segs.data(), segs_bytes);
+        std::memset(h + l.segs_off + segs_bytes, 0, l.items_off - l.segs_off - segs_bytes);
+        std::memcpy(h + l.items_off, wl.item_first.data(), items_bytes);
+        TM_CUDA(cudaMemcpyAsync(d_ws, h, span, cudaMemcpyHostToDevice, st));
+        TM_CUDA(g_staging.mark(dev, slot, st));
+        return TM_OK;
+      }
+    }
+  }
   TM_CUDA(cudaMemsetAsync(d_ws, 0, tms::kStatusBlockBytes, st));
-  if (!wl.segs.empty())
-    TM_CUDA(cudaMemcpyAsync(d_ws + l.segs_off, wl.segs.data(), wl.segs.size() * sizeof(tms::Seg),
-                            cudaMemcpyHostToDevice, st));
-  TM_CUDA(cudaMemcpyAsync(d_ws + l.items_off, wl.item_first.data(),
-                          wl.item_first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+  if (segs_bytes != 0)
+    TM_CUDA(cudaMemcpyAsync(d_ws + l.segs_off, wl.segs.data(), segs_bytes, cudaMemcpyHostToDevice, st));
+  TM_CUDA(cudaMemcpyAsync(d_ws + l.items_off, wl.item_first.data(), items_bytes, cudaMemcpyHostToDevice, st));
   return TM_OK;
 }
 

@@ -92,9 +92,6 @@ __device__ __forceinline__ void bulk_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void consumer_barrier() {
-  asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory");
-}
 
 // How one piece is cut into ring stages.  Destination vectors are 16-byte aligned; `head` bytes
 // before the first aligned destination vector and `rem` bytes after the last full one are copied
@@ -135,7 +132,6 @@ __device__ __forceinline__ bool plan_bulk(const Seg& s, uint8_t* flat, BulkPlan&
 struct RingShared {
   uint64_t full[kRingStages];
   uint64_t empty[kRingStages];
-  unsigned long long red[kConsWarps];
   int abort_flag;
 };
 
@@ -144,19 +140,13 @@ __device__ __forceinline__ void raise_timeout(int* status, RingShared* sh) {
   atomicExch(&sh->abort_flag, 1);
 }
 
-// Sum over the consumer warps of a per-thread value, added to *target by one thread.
-__device__ __forceinline__ void consumer_flush(u64 value, u64* target, RingShared* sh) {
+// Adds a per-thread value, summed over the warp by shuffles, to *target: one atomic per warp.  The
+// consumer warps do not meet at a block barrier for this, so a bucket change never stalls the ring;
+// integer addition mod 2^64 commutes, so the result does not depend on the order of the atomics.
+__device__ __forceinline__ void consumer_flush(u64 value, u64* target) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) value += __shfl_xor_sync(0xffffffffu, value, o);
-  if ((threadIdx.x & 31) == 0) sh->red[threadIdx.x >> 5] = value;
-  consumer_barrier();
-  if (threadIdx.x == 0) {
-    u64 total = 0;
-#pragma unroll
-    for (int w = 0; w < kConsWarps; ++w) total += sh->red[w];
-    if (total != 0) atomicAdd(target, total);
-  }
-  consumer_barrier();
+  if ((threadIdx.x & 31) == 0 && value != 0) atomicAdd(target, value);
 }
 
 // PACK: tensors -> stream with padding and checksums.  Otherwise a plain copy of pieces, direction
@@ -277,7 +267,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
     if (PACK) {
       const uint32_t bucket = segs[first].bucket;
       if (bucket != cur) {   // uniform over the consumers
-        if (cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur, &sh);
+        if (cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur);
         total = 0;
         cur = bucket;
       }
@@ -306,8 +296,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       }
       continue;
     }
-    // After a timeout the consumers keep walking the item list without touching memory, so that
-    // every consumer still meets the others at the checksum barriers.
+    // After a timeout the consumers only walk the rest of the item list, touching no memory.
     if (!ok) continue;
     // bulk piece: head bytes directly, full vectors through the ring, tail (and padding) directly
     if (2 * c < p.head) st2(p.dst - p.head + 2 * c, ld2(p.src - p.head + 2 * c));
@@ -363,7 +352,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       if (2 * gt < p.rem) st2(p.dst + tl + 2 * gt, ld2(p.src + tl + 2 * gt));
     }
   }
-  if (PACK && cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur, &sh);
+  if (PACK && cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur);
 }
 
 // Exercises the bounded wait on purpose: one thread waits for a barrier phase that nobody will ever
