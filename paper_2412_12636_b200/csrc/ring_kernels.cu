@@ -29,6 +29,7 @@ namespace tms {
 constexpr int kRingStages = 3;
 constexpr uint32_t kStageBytes = 32 * 1024;
 constexpr uint32_t kStageVectors = kStageBytes / 16;
+constexpr uint32_t kStageStride = kStageBytes + 128;   // room for the one extra vector of a shifted source
 constexpr int kConsWarps = 8;
 constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kRingThreads = kConsThreads + 64;     // + one producer warp + one store warp
@@ -72,9 +73,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
     if (global_ns() - t0 > limit_ns) return false;
   }
 }
-// Non-multicast 1-D bulk copy global -> this block's shared memory, completion on an mbarrier.
+// 1-D bulk copy global -> this block's own shared memory (single destination block), completion on an mbarrier.
 __device__ __forceinline__ void bulk_g2s(void* smem, const void* g, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+  asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                    smem_u32(smem)),
                "l"(g), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
@@ -123,7 +124,7 @@ __device__ __forceinline__ bool plan_bulk(const Seg& s, uint8_t* flat, BulkPlan&
   p.rem = n & 15;
   p.a = (uint32_t)((uintptr_t)p.src & 15);
   p.sa = p.src - p.a;
-  p.V = kStageVectors - (p.a != 0 ? 1u : 0u);
+  p.V = kStageVectors;
   p.ntiles = (p.nfull + p.V - 1) / p.V;
   p.straight = (p.a == 0);   // the destination is aligned by construction (head bytes are cut off)
   return p.nfull >= kBulkMinVectors;
@@ -191,7 +192,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
         if (cnt > p.V) cnt = p.V;
         const uint32_t bytes = (cnt + extra) * 16u;
         mbar_expect_tx(&sh.full[stage], bytes);
-        bulk_g2s(ring + (size_t)stage * kStageBytes, p.sa + (size_t)t * p.V * 16u, bytes, &sh.full[stage]);
+        bulk_g2s(ring + (size_t)stage * kStageStride, p.sa + (size_t)t * p.V * 16u, bytes, &sh.full[stage]);
         ++issued;
         if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
       }
@@ -231,7 +232,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
         if (p.straight) {
           uint32_t cnt = p.nfull - t * p.V;
           if (cnt > p.V) cnt = p.V;
-          bulk_s2g(p.dst + (size_t)t * p.V * 16u, ring + (size_t)stage * kStageBytes, cnt * 16u);
+          bulk_s2g(p.dst + (size_t)t * p.V * 16u, ring + (size_t)stage * kStageStride, cnt * 16u);
           bulk_commit();
           if (pending >= 0) {
             bulk_wait_read<1>();
@@ -309,7 +310,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       }
       uint32_t cnt = p.nfull - t * p.V;
       if (cnt > p.V) cnt = p.V;
-      const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageBytes);
+      const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageStride);
       const uint32_t vbase = t * p.V;
       uint8_t* d = p.dst + (size_t)vbase * 16u;
       if (p.straight) {
@@ -382,7 +383,7 @@ static int launch_ring(K kernel, const Seg* d_segs, const uint32_t* d_item_first
   int sms = 0;
   int rc = device_sm_count(&sms);
   if (rc != 0) return rc;
-  const size_t smem = (size_t)kRingStages * kStageBytes;
+  const size_t smem = (size_t)kRingStages * kStageStride;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return (int)e;
   uint64_t grid = (uint64_t)sms * tuning().ring_ctas_per_sm;
