@@ -233,7 +233,7 @@ int tm_shard_workspace(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, 
   rc = tm_bounds_u128(n_elems, r, D, &lo, &hi);
   if (rc != TM_OK) return rc;
   // upper bound on pieces: every tensor adds at most two partial pieces to the chunk count
-  const uint64_t chunk = tms::tuning().chunk_bytes;
+  const uint64_t chunk = tms::tuning().shard_chunk_bytes;
   const uint64_t max_segs = (hi - lo) * e / chunk + 2 * n_desc + 2;
   *workspace_bytes = tms::workspace_layout(max_segs, max_segs).total;
   return TM_OK;

@@ -21,8 +21,10 @@ static uint64_t env_u64(const char* name, uint64_t dflt) {
 const Tuning& tuning() {
   static const Tuning t = [] {
     Tuning x;
-    x.chunk_bytes = align_up(env_u64("TM_CHUNK_BYTES", 64 * 1024), 256);
+    x.chunk_bytes = align_up(env_u64("TM_CHUNK_BYTES", 256 * 1024), 256);
     if (x.chunk_bytes > (1ull << 30)) x.chunk_bytes = 1ull << 30;
+    x.shard_chunk_bytes = align_up(env_u64("TM_SHARD_CHUNK_BYTES", 64 * 1024), 256);
+    if (x.shard_chunk_bytes > (1ull << 30)) x.shard_chunk_bytes = 1ull << 30;
     x.small_bytes = env_u64("TM_SMALL_BYTES", 8 * 1024);
     x.group_bytes = env_u64("TM_GROUP_BYTES", 64 * 1024);
     x.group_max = (uint32_t)env_u64("TM_GROUP_MAX", 64);
@@ -173,7 +175,7 @@ int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_
 // d_out.  Pieces after the first of each tensor start on a 256-byte boundary of the output.
 void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
                        uint64_t d_out, tms::WorkList* wl) {
-  const uint64_t chunk = tms::tuning().chunk_bytes;
+  const uint64_t chunk = tms::tuning().shard_chunk_bytes;
   tms::WorkListBuilder builder(wl);
   uint64_t start = 0;  // element index of the tensor's first element in the flat plane
   for (uint64_t k = 0; k < n_desc && start < hi; ++k) {

@@ -75,7 +75,7 @@ extern "C" int tm_shard_extract_static(const tm_desc* plane_descs, uint64_t n_de
   const uint64_t out_bytes = (hi - lo) * e;
   if (out_capacity < out_bytes) return TM_ERR_CAPACITY;
   // refuse oversized requests from the byte count alone, before building any list
-  const uint64_t chunk = tms::tuning().chunk_bytes;
+  const uint64_t chunk = tms::tuning().shard_chunk_bytes;
   const uint64_t min_segs = out_bytes / chunk;
   if (tms::workspace_layout(min_segs, 1).total > TM_STATIC_SCRATCH_BYTES) return TM_ERR_CAPACITY;
   const uint64_t out_addr = (uint64_t)(uintptr_t)d_out;

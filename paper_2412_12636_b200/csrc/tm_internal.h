@@ -47,7 +47,8 @@ class WorkListBuilder {
 };
 
 struct Tuning {
-  uint64_t chunk_bytes;    // largest piece; multiple of 256
+  uint64_t chunk_bytes;    // largest piece of a pack / unpack plan; multiple of 256
+  uint64_t shard_chunk_bytes;  // largest piece of a shard list (smaller: a shard is a fraction of a role)
   uint64_t small_bytes;    // pieces below this share items
   uint64_t group_bytes;    // byte budget of a shared item
   uint32_t group_max;      // piece budget of a shared item

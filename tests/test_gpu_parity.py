@@ -33,10 +33,10 @@ def test_odd_layouts_pack_checksum_unpack(oracle_mod, seed, B):
 
 
 @pytest.mark.parametrize("numel", [1, 2, 7, 8, 9, 127, 128, 129, 4095, 4096, 4097, 32767, 32768, 32769, 65535, 65537,
-                                   3 * 32768 + 5])
+                                   3 * 32768 + 5, 131071, 131072, 131073, 2 * 131072 + 3])
 @pytest.mark.parametrize("misalign", [0, 2, 4, 6, 8, 10, 12, 14])
 def test_single_tensor_every_alignment(oracle_mod, numel, misalign):
-    # bf16 elements: sizes around the vector (16 B), small-piece (8 KiB) and chunk (64 KiB) cuts
+    # bf16 elements: sizes around the vector (16 B), small-piece (8 KiB), ring-stage (32 KiB) and chunk (256 KiB) cuts
     arena = torch.randint(0, 256, (2 * numel + 64,), dtype=torch.uint8, device="cuda",
                           generator=torch.Generator("cuda").manual_seed(numel * 16 + misalign))
     t = arena[misalign:misalign + 2 * numel]
