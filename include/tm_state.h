@@ -157,6 +157,17 @@ int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, ui
                      void* d_out, uint64_t out_capacity, uint64_t* out_elems,
                      void* d_workspace, uint64_t workspace_bytes, void* stream);
 
+/* Shard extract of several planes in one launch (a joiner needs the same [lo, hi) of the fp32
+ * master weights, Adam m and Adam v — §7 "State Synchronization").  `descs` is the concatenation of
+ * the planes' descriptor lists, plane p having plane_n_desc[p] entries; each plane is validated and
+ * sliced exactly as by tm_shard_extract with the same r and D (its own elem_size and element count),
+ * and written contiguously to d_outs[p] (capacity out_capacities[p] bytes).  out_elems (host array of
+ * n_planes entries, may be NULL) receives each plane's hi - lo.  Outputs must not overlap any tensor
+ * or one another.  Workspace: the sum of tm_shard_workspace() over the planes is enough. */
+int tm_shard_extract_planes(const tm_desc* descs, const uint64_t* plane_n_desc, uint32_t n_planes,
+                            uint32_t r, uint32_t D, void* const* d_outs, const uint64_t* out_capacities,
+                            uint64_t* out_elems, void* d_workspace, uint64_t workspace_bytes, void* stream);
+
 /* Shard insert: the inverse of tm_shard_extract (a joiner that fetched its slice of the optimizer
  * state from a peer or from storage — §7 "State Synchronization", the no-redundancy case — puts it
  * into its own flat plane).  Elements [lo, hi) of the plane (same definition and bounds as

@@ -32,6 +32,7 @@ SIGNATURES = {
     "tm_shard_bounds": (_int, [_u64, _u32, _u32, _p, _p]),
     "tm_shard_workspace": (_int, [_p, _u64, _u32, _u32, _p]),
     "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
+    "tm_shard_extract_planes": (_int, [_p, _p, _u32, _u32, _u32, _p, _p, _p, _p, _u64, _p]),
     "tm_shard_insert": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
     "tm_shard_extract_static": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p]),
     "tm_selftest_bounded_wait": (_int, [_p, _u64, _p]),
@@ -161,6 +162,20 @@ def tm_shard_extract(descs, r: int, D: int, d_out: int, out_capacity: int, d_wor
     _check(load_library().tm_shard_extract(arr, len(arr), r, D, d_out, out_capacity, ctypes.byref(n),
                                            d_workspace, workspace_bytes, stream), "tm_shard_extract")
     return n.value
+
+
+def tm_shard_extract_planes(planes, r: int, D: int, d_outs: Sequence[int], out_capacities: Sequence[int],
+                            d_workspace: int, workspace_bytes: int, stream: int) -> List[int]:
+    """`planes` is a list of descriptor lists; returns the number of elements written per plane."""
+    flat = [d for plane in planes for d in plane]
+    arr = make_descs(flat)
+    counts = (_u64 * len(planes))(*[len(p) for p in planes])
+    outs = (_p * len(planes))(*d_outs)
+    caps = (_u64 * len(planes))(*out_capacities)
+    got = (_u64 * len(planes))()
+    _check(load_library().tm_shard_extract_planes(arr, counts, len(planes), r, D, outs, caps, got, d_workspace,
+                                                  workspace_bytes, stream), "tm_shard_extract_planes")
+    return list(got)
 
 
 def tm_shard_insert(descs, r: int, D: int, d_in: int, in_bytes: int, d_workspace: int, workspace_bytes: int,

@@ -3,10 +3,12 @@
 // a CUDA device every operation fails with TM_ERR_CUDA.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "tm_internal.h"
 
@@ -17,6 +19,8 @@ int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_
 void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
                        uint64_t d_out, tms::WorkList* wl);
 int tm_targets_disjoint(const tm_plan* p);
+void tm_shard_append(tms::WorkListBuilder* builder, const tm_desc* descs, uint64_t n_desc, uint32_t e,
+                     uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base);
 
 namespace {
 
@@ -278,6 +282,69 @@ int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, ui
                      uint64_t workspace_bytes, void* stream) {
   return shard_run(plane_descs, n_desc, r, D, d_out, out_capacity, out_elems, d_workspace, workspace_bytes,
                    stream, /*to_tensors=*/false);
+}
+
+int tm_shard_extract_planes(const tm_desc* descs, const uint64_t* plane_n_desc, uint32_t n_planes, uint32_t r,
+                            uint32_t D, void* const* d_outs, const uint64_t* out_capacities,
+                            uint64_t* out_elems, void* d_workspace, uint64_t workspace_bytes, void* stream) {
+  if (descs == nullptr || plane_n_desc == nullptr || n_planes == 0 || d_outs == nullptr ||
+      out_capacities == nullptr)
+    return TM_ERR_ARG;
+  if (d_workspace == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+  struct PlaneInfo { const tm_desc* d; uint64_t n; uint32_t e; uint64_t lo, hi; };
+  std::vector<PlaneInfo> planes(n_planes);
+  const tm_desc* cursor = descs;
+  uint64_t base = ~0ull;
+  for (uint32_t p = 0; p < n_planes; ++p) {
+    PlaneInfo& pi = planes[p];
+    pi.d = cursor;
+    pi.n = plane_n_desc[p];
+    uint64_t n_elems = 0;
+    int rc = tm_shard_validate(pi.d, pi.n, r, D, &pi.e, &n_elems);
+    if (rc != TM_OK) return rc;
+    rc = tm_bounds_u128(n_elems, r, D, &pi.lo, &pi.hi);
+    if (rc != TM_OK) return rc;
+    cursor += pi.n;
+    if (pi.hi == pi.lo) continue;
+    if (d_outs[p] == nullptr) return TM_ERR_ARG;
+    if (((uintptr_t)d_outs[p] & 1) != 0) return TM_ERR_ALIGN;
+    if (out_capacities[p] < (pi.hi - pi.lo) * pi.e) return TM_ERR_CAPACITY;
+    base = std::min(base, (uint64_t)(uintptr_t)d_outs[p]);
+  }
+  // no output may overlap a tensor of any plane, nor another output
+  const uint64_t n_total = (uint64_t)(cursor - descs);
+  for (uint32_t p = 0; p < n_planes; ++p) {
+    if (planes[p].hi == planes[p].lo) continue;
+    const uint64_t o = (uint64_t)(uintptr_t)d_outs[p], ob = (planes[p].hi - planes[p].lo) * planes[p].e;
+    for (uint64_t k = 0; k < n_total; ++k)
+      if (ranges_overlap((uint64_t)(uintptr_t)descs[k].ptr, descs[k].nbytes, o, ob)) return TM_ERR_OVERLAP;
+    for (uint32_t q = p + 1; q < n_planes; ++q) {
+      if (planes[q].hi == planes[q].lo) continue;
+      if (ranges_overlap(o, ob, (uint64_t)(uintptr_t)d_outs[q], (planes[q].hi - planes[q].lo) * planes[q].e))
+        return TM_ERR_OVERLAP;
+    }
+  }
+  if (out_elems != nullptr)
+    for (uint32_t p = 0; p < n_planes; ++p) out_elems[p] = planes[p].hi - planes[p].lo;
+  if (base == ~0ull) return TM_OK;   // every shard is empty
+  tms::WorkList wl;
+  tms::WorkListBuilder builder(&wl);
+  for (uint32_t p = 0; p < n_planes; ++p)
+    if (planes[p].hi != planes[p].lo)
+      tm_shard_append(&builder, planes[p].d, planes[p].n, planes[p].e, planes[p].lo, planes[p].hi,
+                      (uint64_t)(uintptr_t)d_outs[p], base);
+  builder.finish();
+  const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
+  if (workspace_bytes < l.total) return TM_ERR_CAPACITY;
+  int rc = upload_worklist(wl, l, (uint8_t*)d_workspace, (cudaStream_t)stream);
+  if (rc != TM_OK) return rc;
+  const uint8_t* ws = (const uint8_t*)d_workspace;
+  auto copy_fn = tms::tuning().use_ring ? tms::launch_copy_ring : tms::launch_copy;
+  int err = copy_fn((const tms::Seg*)(ws + l.segs_off), (const uint32_t*)(ws + l.items_off),
+                    (uint32_t)wl.n_items(), (uint8_t*)(uintptr_t)base, /*to_tensors=*/false,
+                    (int*)d_workspace, stream);
+  return err == 0 ? TM_OK : cuda_fail(err);
 }
 
 int tm_shard_insert(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, const void* d_in,

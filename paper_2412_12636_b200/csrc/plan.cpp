@@ -171,12 +171,12 @@ int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_
   return TM_OK;
 }
 
-// Work list that gathers elements [lo, hi) of the plane into a contiguous output at address
-// d_out.  Pieces after the first of each tensor start on a 256-byte boundary of the output.
-void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
-                       uint64_t d_out, tms::WorkList* wl) {
+// Appends the pieces that gather elements [lo, hi) of one plane into a contiguous output at address
+// d_out; piece offsets are relative to `flat_base` (<= d_out).  Pieces after the first of each
+// tensor start on a 256-byte boundary of the output.
+void tm_shard_append(tms::WorkListBuilder* builder, const tm_desc* descs, uint64_t n_desc, uint32_t e,
+                     uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base) {
   const uint64_t chunk = tms::tuning().shard_chunk_bytes;
-  tms::WorkListBuilder builder(wl);
   uint64_t start = 0;  // element index of the tensor's first element in the flat plane
   for (uint64_t k = 0; k < n_desc && start < hi; ++k) {
     const uint64_t count = descs[k].nbytes / e;
@@ -193,12 +193,12 @@ void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64
         len = std::min(len, remaining);
         Seg s;
         s.tensor = tensor;
-        s.off = out;
+        s.off = (d_out - flat_base) + out;
         s.nbytes = (uint32_t)len;
         s.pad = 0;
         s.bucket = 0;
         s.word0 = 0;
-        builder.add(s);
+        builder->add(s);
         tensor += len;
         out += len;
         remaining -= len;
@@ -206,6 +206,13 @@ void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64
     }
     start += count;
   }
+}
+
+// Work list for one plane, offsets relative to d_out.
+void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
+                       uint64_t d_out, tms::WorkList* wl) {
+  tms::WorkListBuilder builder(wl);
+  tm_shard_append(&builder, descs, n_desc, e, lo, hi, d_out, d_out);
   builder.finish();
 }
 

@@ -80,6 +80,40 @@ class ShardExtractor:
                                        self.workspace.numel(), _stream_handle(stream))
 
 
+class MultiShardExtractor:
+    """Shard r of D of several planes (each with its own element size) in one launch."""
+
+    def __init__(self, planes: Sequence[Sequence[Tuple[int, int, int, int]]], r: int, D: int, device="cuda"):
+        import ctypes
+        self.device = torch.device(device)
+        self.r, self.D, self.n_planes = r, D, len(planes)
+        self._descs = binding.make_descs([d for plane in planes for d in plane])
+        self._counts = (ctypes.c_uint64 * self.n_planes)(*[len(p) for p in planes])
+        self.out_bytes = []
+        ws = 0
+        for plane in planes:
+            e = plane[0][2]
+            lo, hi = binding.tm_shard_bounds(sum(d[1] for d in plane) // e, r, D)
+            self.out_bytes.append((hi - lo) * e)
+            ws += binding.tm_shard_workspace(plane, r, D)
+        self.workspace = torch.empty(ws, dtype=torch.uint8, device=self.device)
+        self._got = (ctypes.c_uint64 * self.n_planes)()
+
+    def alloc_outs(self):
+        return [torch.empty(n, dtype=torch.uint8, device=self.device) for n in self.out_bytes]
+
+    def extract(self, outs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None):
+        import ctypes
+        ptrs = (ctypes.c_void_p * self.n_planes)(*[o.data_ptr() for o in outs])
+        caps = (ctypes.c_uint64 * self.n_planes)(*[o.numel() * o.element_size() for o in outs])
+        L = binding.load_library()
+        binding._check(L.tm_shard_extract_planes(self._descs, self._counts, self.n_planes, self.r, self.D, ptrs,
+                                                 caps, self._got, self.workspace.data_ptr(),
+                                                 self.workspace.numel(), _stream_handle(stream)),
+                       "tm_shard_extract_planes")
+        return list(self._got)
+
+
 class WaveMover:
     """The same role cut into waves of whole buckets (see waves.py), one plan per wave.
 

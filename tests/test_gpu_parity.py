@@ -253,3 +253,30 @@ def test_expired_device_wait_is_reported_not_hung():
     binding.tm_checksum(data.data_ptr(), 8 << 16, 8 << 16, out.data_ptr(), s)
     torch.cuda.synchronize()
     assert int(G.u64(out)[0]) == (1 << 32)               # c * n^2 with c = 1, n = 2^16
+
+
+def test_multi_plane_shard_extract_matches_oracle_per_plane(oracle_mod):
+    from paper_2412_12636_b200.mover import MultiShardExtractor
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    adv = layouts.materialize_adversarial(layouts.adversarial_specs(300, max_log2=16), "cuda", seed=5)
+    cases = [
+        (state, [state.plane_indices(p) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)], 1, 2),
+        (adv, [adv.elem_size_indices(e) for e in (4, 2, 8)], 17, 64),        # mixed element sizes in one call
+        (adv, [adv.elem_size_indices(e) for e in (8, 4)], 10 ** 9 - 1, 10 ** 9),   # D > N: one-element shards
+        (adv, [adv.elem_size_indices(e) for e in (8, 4)], 0, 10 ** 9),             # D > N: empty shards, no launch
+    ]
+    for st, planes, r, D in cases:
+        ms = MultiShardExtractor([st.descs_of(idx) for idx in planes], r, D)
+        bufs = [G.guarded(n) for n in ms.out_bytes]
+        got = ms.extract([b[1] for b in bufs])
+        torch.cuda.synchronize()
+        if any(ms.out_bytes):
+            assert binding.tm_workspace_status(ms.workspace.data_ptr(), torch.cuda.current_stream().cuda_stream) == 0
+        for idx, (whole, out), n_el, nbytes in zip(planes, bufs, got, ms.out_bytes):
+            e = st.specs[idx[0]].elem_size
+            host = [st.host_bytes(i) for i in idx]
+            expect = oracle_mod.shard(host, [h.size for h in host], e, r, D)
+            assert n_el * e == expect.size == nbytes
+            assert np.array_equal(out.cpu().numpy(), expect)
+            assert G.guards_intact(whole, nbytes)
