@@ -475,7 +475,7 @@ def run_e2e(args, role):
     torch.cuda.synchronize()
     compute = torch.cuda.current_stream()
     up, down = torch.cuda.Stream(), torch.cuda.Stream()
-    wave_bytes = max(role.bucket_bytes, 1 << 30)
+    wave_bytes = max(role.bucket_bytes, int(os.environ.get("TM_BENCH_WAVE_MB", "1024")) << 20)
     wm = WaveMover(state.descs(), role.bucket_bytes, wave_bytes)
     torch.cuda.synchronize()
     dev_bytes = [layouts.tensor_bytes(t) for t in state.tensors]

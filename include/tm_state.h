@@ -136,6 +136,16 @@ int tm_state_pack(const tm_plan* plan, void* d_buckets, uint64_t capacity,
  * must not overlap the packed buffer or one another. */
 int tm_state_unpack(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, void* stream);
 
+/* Unpack and verify in one pass (joiner side: checking the received buckets and overwriting the
+ * sandbox-warmed state are both part of "State Synchronization", §7; the paper has no integrity check,
+ * the checksum is this library's).  Does what tm_state_unpack does and, while the buckets stream
+ * through, accumulates the checksum of every bucket exactly as tm_checksum(d_buckets, T, B) defines it
+ * — over the bytes as received, padding included — into d_checksums (n_buckets uint64, 8-byte
+ * aligned, required).  The caller compares them with the sender's after synchronising; the tensors
+ * have been written by then, so a mismatch means the unpacked state must be discarded. */
+int tm_state_unpack_verify(const tm_plan* plan, const void* d_buckets, uint64_t nbytes,
+                           uint64_t* d_checksums, void* stream);
+
 /* Host helper: floor shard bounds lo = floor(r*N/D), hi = floor((r+1)*N/D) in 128-bit arithmetic. */
 int tm_shard_bounds(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
 

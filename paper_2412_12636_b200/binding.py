@@ -29,6 +29,7 @@ SIGNATURES = {
     "tm_plan_destroy": (None, [_p]),
     "tm_state_pack": (_int, [_p, _p, _u64, _p, _p]),
     "tm_state_unpack": (_int, [_p, _p, _u64, _p]),
+    "tm_state_unpack_verify": (_int, [_p, _p, _u64, _p, _p]),
     "tm_shard_bounds": (_int, [_u64, _u32, _u32, _p, _p]),
     "tm_shard_workspace": (_int, [_p, _u64, _u32, _u32, _p]),
     "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
@@ -139,6 +140,11 @@ def tm_state_pack(plan: Plan, d_buckets: int, capacity: int, d_checksums: Option
 
 def tm_state_unpack(plan: Plan, d_buckets: int, nbytes: int, stream: int) -> None:
     _check(load_library().tm_state_unpack(plan.handle, d_buckets, nbytes, stream), "tm_state_unpack")
+
+
+def tm_state_unpack_verify(plan: Plan, d_buckets: int, nbytes: int, d_checksums: int, stream: int) -> None:
+    _check(load_library().tm_state_unpack_verify(plan.handle, d_buckets, nbytes, d_checksums, stream),
+           "tm_state_unpack_verify")
 
 
 def tm_shard_bounds(n_elems: int, r: int, D: int) -> Tuple[int, int]:

@@ -221,6 +221,26 @@ int tm_state_unpack(const tm_plan* plan, const void* d_buckets, uint64_t nbytes,
   return e == 0 ? TM_OK : cuda_fail(e);
 }
 
+int tm_state_unpack_verify(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, uint64_t* d_checksums,
+                           void* stream) {
+  if (plan == nullptr || d_buckets == nullptr || d_checksums == nullptr) return TM_ERR_ARG;
+  if (plan->d_workspace == nullptr) return TM_ERR_STATE;
+  if (((uintptr_t)d_buckets & 255) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
+  if (nbytes < plan->total_bytes) return TM_ERR_CAPACITY;
+  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
+  for (const tm_desc& d : plan->descs)
+    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
+  if (plan->targets_disjoint == 0) plan->targets_disjoint = tm_targets_disjoint(plan);
+  if (plan->targets_disjoint < 0) return TM_ERR_OVERLAP;
+  TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), (cudaStream_t)stream));
+  const uint8_t* ws = plan->d_workspace;
+  int e = tms::launch_unpack_verify_ring((const tms::Seg*)(ws + plan->ws_layout.segs_off),
+                                         (const uint32_t*)(ws + plan->ws_layout.items_off),
+                                         (uint32_t)plan->work.n_items(), (uint8_t*)const_cast<void*>(d_buckets),
+                                         (unsigned long long*)d_checksums, (int*)plan->d_workspace, stream);
+  return e == 0 ? TM_OK : cuda_fail(e);
+}
+
 int tm_shard_bounds(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi) {
   if (lo == nullptr || hi == nullptr) return TM_ERR_ARG;
   return tm_bounds_u128(n_elems, r, D, lo, hi);

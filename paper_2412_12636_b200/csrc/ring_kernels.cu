@@ -151,8 +151,10 @@ __device__ __forceinline__ void consumer_flush(u64 value, u64* target) {
 }
 
 // PACK: tensors -> stream with padding and checksums.  Otherwise a plain copy of pieces, direction
-// given by TO_TENSORS (PACK implies TO_TENSORS == false).
-template <bool PACK, bool TO_TENSORS>
+// given by TO_TENSORS (PACK implies TO_TENSORS == false).  VERIFY (with TO_TENSORS): the unpack also
+// accumulates the per-bucket checksums of the stream it reads — data and padding bytes as they
+// arrived — so that a receiver checks and scatters in one pass over the buckets.
+template <bool PACK, bool TO_TENSORS, bool VERIFY>
 __global__ void __launch_bounds__(kRingThreads, 1)
 ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
             uint8_t* __restrict__ flat, u64* __restrict__ checksums, int* __restrict__ status) {
@@ -265,7 +267,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
   bool ok = true;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t first = item_first[item], last = item_first[item + 1];
-    if (PACK) {
+    if (PACK || VERIFY) {
       const uint32_t bucket = segs[first].bucket;
       if (bucket != cur) {   // uniform over the consumers
         if (cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur);
@@ -293,6 +295,11 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
           uint8_t* t = reinterpret_cast<uint8_t*>(s.tensor);
           uint8_t* f = flat + s.off;
           copy_piece(TO_TENSORS ? t : f, TO_TENSORS ? f : t, s.nbytes, g, G);
+          if (VERIFY) {   // the piece's span of the stream, padding included, in aligned vectors
+            const uint32_t nvec = (s.nbytes + s.pad) >> 4;
+            for (uint32_t v = g; v < nvec; v += G) ck.add(ld16_cached(f + (size_t)v * 16u), v);
+            total += ck.finish(s.word0);
+          }
         }
       }
       continue;
@@ -313,17 +320,20 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageStride);
       const uint32_t vbase = t * p.V;
       uint8_t* d = p.dst + (size_t)vbase * 16u;
+      // VERIFY: the stream piece starts 256-byte aligned, so stage vector v is stream vector vbase + v
       if (p.straight) {
-        if (PACK) {   // the store thread moves the data; only the checksum is left to do
+        if (PACK || VERIFY) {   // the store thread moves the data; only the checksum is left to do
 #pragma unroll 4
           for (uint32_t v = c; v < cnt; v += kConsThreads) ck.add(sp[v], vbase + v);
         }
       } else {
 #pragma unroll 2
         for (uint32_t v = c; v < cnt; v += kConsThreads) {
-          const uint4 x = shift_pair(sp[v], sp[v + 1], ws, bs);
+          const uint4 lo = sp[v];
+          const uint4 x = shift_pair(lo, sp[v + 1], ws, bs);
           st16(d + (size_t)v * 16u, x);
           if (PACK) ck.add(x, vbase + v);
+          if (VERIFY) ck.add(lo, vbase + v);
         }
       }
       __syncwarp();
@@ -351,9 +361,15 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       const size_t tl = (size_t)p.nfull * 16u;
       const uint32_t gt = kConsThreads - 1 - c;
       if (2 * gt < p.rem) st2(p.dst + tl + 2 * gt, ld2(p.src + tl + 2 * gt));
+      if (VERIFY) {   // stream vectors behind the ring's share: end of the data and the padding
+        const uint8_t* f = flat + s0.off;
+        const uint32_t nvec = (s0.nbytes + s0.pad) >> 4;
+        for (uint32_t v = p.nfull + c; v < nvec; v += kConsThreads) ck.add(ld16_cached(f + (size_t)v * 16u), v);
+        total += ck.finish(s0.word0);
+      }
     }
   }
-  if (PACK && cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur);
+  if ((PACK || VERIFY) && cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur);
 }
 
 // Exercises the bounded wait on purpose: one thread waits for a barrier phase that nobody will ever
@@ -397,15 +413,21 @@ static int launch_ring(K kernel, const Seg* d_segs, const uint32_t* d_item_first
 
 int launch_pack_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
                      unsigned long long* d_checksums, int* d_status, void* stream) {
-  return launch_ring(ring_kernel<true, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
+  return launch_ring(ring_kernel<true, false, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
                      stream);
 }
 
 int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
                      bool to_tensors, int* d_status, void* stream) {
   if (to_tensors)
-    return launch_ring(ring_kernel<false, true>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
-  return launch_ring(ring_kernel<false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
+    return launch_ring(ring_kernel<false, true, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
+  return launch_ring(ring_kernel<false, false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
+}
+
+int launch_unpack_verify_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
+                              unsigned long long* d_checksums, int* d_status, void* stream) {
+  return launch_ring(ring_kernel<false, true, true>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
+                     stream);
 }
 
 }  // namespace tms

@@ -80,6 +80,8 @@ int launch_pack_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n
                      unsigned long long* d_checksums, int* d_status, void* stream);
 int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
                      bool to_tensors, int* d_status, void* stream);
+int launch_unpack_verify_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
+                              unsigned long long* d_checksums, int* d_status, void* stream);
 int launch_wait_selftest(int* d_status, unsigned long long limit_ns, void* stream);
 int launch_checksum(const uint8_t* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
                     unsigned long long* d_checksums, void* stream);

@@ -42,6 +42,12 @@ class RoleMover:
         binding.tm_state_unpack(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
                                 _stream_handle(stream))
 
+    def unpack_verify(self, buckets: torch.Tensor, checksums: torch.Tensor,
+                      stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Unpack and, in the same pass, the per-bucket checksums of the buckets as received."""
+        binding.tm_state_unpack_verify(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
+                                       checksums.data_ptr(), _stream_handle(stream))
+
     def checksum(self, buckets: torch.Tensor, checksums: torch.Tensor,
                  stream: Optional[torch.cuda.Stream] = None) -> None:
         binding.tm_checksum(buckets.data_ptr(), self.total_bytes, self.bucket_bytes, checksums.data_ptr(),

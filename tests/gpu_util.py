@@ -78,6 +78,31 @@ def check_pack_against_oracle(oracle, state: layouts.RoleState, bucket_bytes: Op
     else:
         for k, e in enumerate(exp_tensors):
             assert np.array_equal(target.host_bytes(k), e), f"tensor {k} differs after unpack"
+    # unpack + verify in one pass: same tensors, and the checksums of the stream as received — also
+    # when a padding byte (which unpack ignores) arrives corrupted
+    received = buckets.clone()
+    covered = np.zeros(exp_stream.size, dtype=bool)
+    off = mover.plan.offsets()
+    for o, spec in zip(off, state.specs):
+        covered[o:o + spec.nbytes] = True
+    pad_positions = np.flatnonzero(~covered)
+    if pad_positions.size:
+        received[int(pad_positions[pad_positions.size // 2])] = 0x5A
+    exp_received = oracle.checksum(received.cpu().numpy(), B)
+    target2 = layouts.blank_like(state)
+    tm2 = RoleMover(target2.descs(), B)
+    got_cks = tm2.alloc_checksums()
+    tm2.unpack_verify(received, got_cks)
+    torch.cuda.synchronize()
+    assert tm2.status() == 0
+    assert np.array_equal(u64(got_cks), exp_received)
+    if pad_positions.size:
+        assert not np.array_equal(exp_received, exp_cks)
+    if target2.arena is not None:
+        assert torch.equal(target2.arena, target.arena)
+    else:
+        for a, b in zip(target2.tensors, target.tensors):
+            assert torch.equal(layouts.tensor_bytes(a), layouts.tensor_bytes(b))
     return mover, buckets, exp_stream
 
 

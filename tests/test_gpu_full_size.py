@@ -50,12 +50,18 @@ def check_stream_structure_on_device(state, off, buckets, total):
     assert not bool(buckets[pos:total].any())
 
 
-def check_unpack_on_device(state, buckets, B):
+def check_unpack_on_device(state, buckets, B, expect_cks=None):
     target = layouts.blank_like(state)
     um = RoleMover(target.descs(), B)
-    um.unpack(buckets)
+    if expect_cks is None:
+        um.unpack(buckets)
+    else:                                   # unpack + verify in one pass
+        got = um.alloc_checksums()
+        um.unpack_verify(buckets, got)
     torch.cuda.synchronize()
     assert um.status() == 0
+    if expect_cks is not None:
+        assert np.array_equal(G.u64(got), expect_cks)
     if target.arena is not None:
         base_s, base_t = state.arena.data_ptr(), target.arena.data_ptr()
         pos = 0
@@ -109,6 +115,8 @@ def test_full_size_role_configs(oracle_mod, idx):
     check_stream_structure_on_device(state, off, buckets, mover.total_bytes)
     target = check_unpack_on_device(state, buckets, cfg.bucket_bytes)
     del target
+    target = check_unpack_on_device(state, buckets, cfg.bucket_bytes, expect_cks=cks)
+    del target
     expect_elems = {1: 68_753_024, 2: 31_375_488, 3: 44_571_307}[idx]
     for plane in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V):
         out = check_shard_sampled(oracle_mod, state, state.plane_indices(plane), cfg.shard_r, cfg.shard_D)
@@ -144,6 +152,7 @@ def test_adversarial_20000_tensors_single_launch(oracle_mod):
     off = check_sampled_buckets(oracle_mod, state, mover, buckets, cks, sample)
     check_stream_structure_on_device(state, off, buckets, mover.total_bytes)
     check_unpack_on_device(state, buckets, B)
+    check_unpack_on_device(state, buckets, B, expect_cks=cks)
     del buckets
     # shard extract for every r of 64 over the fp32 subset: exact union coverage, oracle on samples
     idx = state.elem_size_indices(4)
