@@ -12,7 +12,7 @@ import json
 import torch
 
 from . import binding, layouts
-from .mover import RoleMover, ShardExtractor
+from .mover import MultiShardExtractor, RoleMover
 
 
 def main() -> None:
@@ -29,24 +29,25 @@ def main() -> None:
     mover = RoleMover(state.descs(), cfg.bucket_bytes)
     unmover = RoleMover(target.descs(), cfg.bucket_bytes)
     buckets, fused, alone = mover.alloc_buckets(), mover.alloc_checksums(), mover.alloc_checksums()
-    shards = []
-    for plane in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V):
-        ex = ShardExtractor(target.descs_of(target.plane_indices(plane)), cfg.shard_r, cfg.shard_D)
-        shards.append((ex, ex.alloc_out()))
-    for _ in range(args.reps):
+    planes = [target.descs_of(target.plane_indices(p)) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)]
+    multi = MultiShardExtractor(planes, cfg.shard_r, cfg.shard_D)
+    outs = multi.alloc_outs()
+    received = mover.alloc_checksums()
+    for _ in range(args.reps):          # launch order per repetition: pack, checksum, unpack, unpack_verify, shard
         mover.pack(buckets, fused)
         mover.checksum(buckets, alone)
         unmover.unpack(buckets)
-        for ex, out in shards:
-            ex.extract(out)
+        unmover.unpack_verify(buckets, received)
+        multi.extract(outs)
     torch.cuda.synchronize()
-    assert torch.equal(fused, alone) and mover.status() == 0
+    assert torch.equal(fused, alone) and torch.equal(fused, received) and mover.status() == 0
     print(json.dumps({"workload": cfg.name, "state_bytes": state.state_bytes, "stream_bytes": mover.total_bytes,
                       "n_buckets": mover.n_buckets,
                       "algorithmic_bytes": {"pack": state.state_bytes + mover.total_bytes + 8 * mover.n_buckets,
                                             "checksum": mover.total_bytes + 8 * mover.n_buckets,
                                             "unpack": 2 * state.state_bytes,
-                                            "shard_per_plane": [2 * ex.out_bytes for ex, _ in shards]},
+                                            "unpack_verify": 2 * state.state_bytes + 8 * mover.n_buckets,
+                                            "shard_three_planes": 2 * sum(multi.out_bytes)},
                       "launches": binding.tm_launch_count()}))
 
 
