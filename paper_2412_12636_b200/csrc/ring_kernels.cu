@@ -310,7 +310,8 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
     if (2 * c < p.head) st2(p.dst - p.head + 2 * c, ld2(p.src - p.head + 2 * c));
     const uint32_t ws = p.a >> 2, bs = (p.a & 3) * 8;
     for (uint32_t t = 0; t < p.ntiles; ++t) {
-      if (!mbar_wait(&sh.full[stage], phase, abort_flag)) {
+      // the vote keeps the warp together: either all of its lanes go on or none does
+      if (!__all_sync(0xffffffffu, mbar_wait(&sh.full[stage], phase, abort_flag))) {
         raise_timeout(status, &sh);
         ok = false;
         break;
