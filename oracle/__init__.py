@@ -39,23 +39,46 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+def _configure(L: ctypes.CDLL) -> ctypes.CDLL:
+    L.oracle_layout.argtypes = [_p, _u64, _u64, _p, _p, _p]
+    L.oracle_checksum.argtypes = [_p, _u64, _u64, _p]
+    L.oracle_pack.argtypes = [_p, _p, _u64, _u64, _p, _u64, _p]
+    L.oracle_pack_range.argtypes = [_p, _p, _u64, _u64, _u64, _p]
+    L.oracle_unpack.argtypes = [_p, _p, _u64, _p, _u64]
+    L.oracle_shard_bounds.argtypes = [_u64, _u32, _u32, _p, _p]
+    L.oracle_shard.argtypes = [_p, _p, _u64, _u32, _u32, _u32, _p, _u64, _p]
+    L.oracle_shard_insert.argtypes = [_p, _p, _u64, _u32, _u32, _u32, _p, _u64, _p]
+    for name in ("oracle_layout", "oracle_checksum", "oracle_pack", "oracle_pack_range",
+                 "oracle_unpack", "oracle_shard_bounds", "oracle_shard", "oracle_shard_insert"):
+        getattr(L, name).restype = ctypes.c_int
+    return L
+
+
 def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(build())
-        L.oracle_layout.argtypes = [_p, _u64, _u64, _p, _p, _p]
-        L.oracle_checksum.argtypes = [_p, _u64, _u64, _p]
-        L.oracle_pack.argtypes = [_p, _p, _u64, _u64, _p, _u64, _p]
-        L.oracle_pack_range.argtypes = [_p, _p, _u64, _u64, _u64, _p]
-        L.oracle_unpack.argtypes = [_p, _p, _u64, _p, _u64]
-        L.oracle_shard_bounds.argtypes = [_u64, _u32, _u32, _p, _p]
-        L.oracle_shard.argtypes = [_p, _p, _u64, _u32, _u32, _u32, _p, _u64, _p]
-        L.oracle_shard_insert.argtypes = [_p, _p, _u64, _u32, _u32, _u32, _p, _u64, _p]
-        for name in ("oracle_layout", "oracle_checksum", "oracle_pack", "oracle_pack_range",
-                     "oracle_unpack", "oracle_shard_bounds", "oracle_shard", "oracle_shard_insert"):
-            getattr(L, name).restype = ctypes.c_int
-        _lib = L
+        _lib = _configure(ctypes.CDLL(build()))
     return _lib
+
+
+class use_library:
+    """Context manager that makes every function of this module call another build of the oracle
+    (used by the mutation test, which plants mistakes in copies of tm_oracle.cpp to show that the
+    pins catch them)."""
+
+    def __init__(self, path: str):
+        self.path = path
+
+    def __enter__(self):
+        global _lib
+        self._saved = lib()
+        _lib = _configure(ctypes.CDLL(self.path))
+        return self
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self._saved
+        return False
 
 
 def _check(rc: int, what: str) -> None:
