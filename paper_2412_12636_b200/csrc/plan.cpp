@@ -137,7 +137,7 @@ int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bu
   builder.finish();
   p->total_bytes = align256(pos);
   p->n_buckets = (p->total_bytes + bucket_bytes - 1) / bucket_bytes;
-  if (p->work.segs.size() >= (1ull << 32)) return TM_ERR_ARG;
+  if (p->work.segs.size() >= (1ull << 32) - (1u << 20)) return TM_ERR_ARG;   // piece and item indices are 32-bit
   p->ws_layout = tms::workspace_layout(p->work.segs.size(), p->work.n_items());
   return TM_OK;
 }
