@@ -134,3 +134,15 @@ def test_no_cpu_fallback_without_a_gpu(lib):
         binding.tm_checksum(host.ctypes.data & ~15, 512, 256, out.ctypes.data, 0)
     assert e.value.status == binding.TM_ERR_CUDA
     assert binding.tm_launch_count() == before and not out.any()
+
+
+def test_header_is_plain_c_and_library_links_from_c(lib, tmp_path):
+    import subprocess
+    exe = tmp_path / "c_abi_check"
+    libdir = os.path.dirname(binding.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                    os.path.join(ROOT, "tests", "c_abi_check.c"), "-o", str(exe), "-L", libdir, "-ltm_state",
+                    f"-Wl,-rpath,{libdir}"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, (out.returncode, out.stdout, out.stderr)
+    assert "c abi ok, 0 launches" in out.stdout
