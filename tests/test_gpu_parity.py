@@ -280,3 +280,32 @@ def test_multi_plane_shard_extract_matches_oracle_per_plane(oracle_mod):
             assert n_el * e == expect.size == nbytes
             assert np.array_equal(out.cpu().numpy(), expect)
             assert G.guards_intact(whole, nbytes)
+
+
+def test_two_streams_run_independent_plans_concurrently(oracle_mod):
+    specs_a = layouts.adversarial_specs(600, max_log2=17)
+    a = layouts.materialize_adversarial(specs_a, "cuda", seed=21)
+    b = layouts.materialize(layouts.role_config(0), "cuda")
+    exp_a, cks_a = oracle_mod.pack(G.host_tensors(a), 1 << 20)
+    exp_b, cks_b = oracle_mod.pack(G.host_tensors(b), 1 << 20)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    ma, mb = RoleMover(a.descs(), 1 << 20, stream=s1), RoleMover(b.descs(), 1 << 20, stream=s2)
+    ba, bb = ma.alloc_buckets(), mb.alloc_buckets()
+    ca, cb = ma.alloc_checksums(), mb.alloc_checksums()
+    ta, tb = layouts.blank_like(a), layouts.blank_like(b)
+    ua, ub = RoleMover(ta.descs(), 1 << 20, stream=s1), RoleMover(tb.descs(), 1 << 20, stream=s2)
+    torch.cuda.synchronize()
+    for _ in range(5):                       # interleave enqueues on the two streams
+        ma.pack(ba, ca, stream=s1)
+        mb.pack(bb, cb, stream=s2)
+        ua.unpack(ba, stream=s1)
+        ub.unpack(bb, stream=s2)
+    torch.cuda.synchronize()
+    assert np.array_equal(ba.cpu().numpy(), exp_a) and np.array_equal(G.u64(ca), cks_a)
+    assert np.array_equal(bb.cpu().numpy(), exp_b) and np.array_equal(G.u64(cb), cks_b)
+    for k in range(0, len(a.tensors), 37):
+        assert np.array_equal(ta.host_bytes(k), a.host_bytes(k))
+    for k in range(len(b.tensors)):
+        assert np.array_equal(tb.host_bytes(k), b.host_bytes(k))
+    assert ma.status(s1) == 0 and mb.status(s2) == 0
