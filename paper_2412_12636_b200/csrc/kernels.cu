@@ -1,6 +1,10 @@
-// sm_100a kernels of the role-state mover: fused pack + checksum, generic piece copy (unpack and
-// shard extract) and stand-alone checksum.  Everything here is HBM-bound byte movement with one
-// 64-bit multiply-add per 8 bytes; there is no contraction, so no tensor cores.
+// Register-path kernels of the role-state mover for sm_100a: the stand-alone checksum
+// (checksum_kernel, the one every tm_checksum call runs), and pack_kernel / copy_kernel — the
+// load/store versions of pack, unpack and shard copy.  The main path of pack, unpack and shard
+// extract is the bulk-copy ring in ring_kernels.cu; pack_kernel / copy_kernel run when
+// TM_USE_RING=0 is set (for A/B measurement) and copy_kernel serves tm_shard_extract_static.
+// Everything here is HBM-bound byte movement with one 64-bit multiply-add per 8 bytes; there is no
+// contraction, so no tensor cores.
 //
 // Work distribution: a persistent grid walks the item list with a grid stride.  An item with one
 // piece is copied by the whole block; an item with several small pieces gives one warp per piece.
