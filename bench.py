@@ -373,6 +373,9 @@ def run_ours(args) -> None:
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    if not os.path.exists(binding.LIB_PATH) and rank == 0:
+        from paper_2412_12636_b200 import build as lib_build     # in-tree build; not a fallback path
+        lib_build.build()
     binding.load_library()
     torch.cuda.set_device(local_rank)
     if world > 1:

@@ -17,3 +17,10 @@ def oracle_mod():
     import oracle
     oracle.build()
     return oracle
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The C-ABI library is built in-tree before any test uses it (a no-op when it is up to date)."""
+    from paper_2412_12636_b200 import build
+    build.build()
