@@ -146,6 +146,19 @@ class WaveMover:
             self.movers.append(RoleMover(part_descs, bucket_bytes, device, stream))
             self.tensor_ranges.append((w.parts[0].tensor, w.parts[-1].tensor + 1))
 
+    def wave_bytes(self, i: int) -> int:
+        return self.waves[i].stream_end - self.waves[i].stream_begin
+
+    def pack_wave_into(self, i: int, slot: torch.Tensor, checksums: Optional[torch.Tensor],
+                       stream: Optional[torch.cuda.Stream] = None) -> int:
+        """Packs wave i into a staging slot (any 256-byte-aligned buffer of at least wave_bytes(i)
+        bytes) — the bounded-channel mode: the caller ships the slot and reuses it for a later wave.
+        `checksums` is the full per-bucket array of the role.  Returns the bytes written."""
+        w = self.waves[i]
+        cks = None if checksums is None else checksums[w.first_bucket:w.first_bucket + w.n_buckets]
+        self.movers[i].pack(slot, cks, stream)
+        return w.stream_end - w.stream_begin
+
     def pack_wave(self, i: int, buckets: torch.Tensor, checksums: Optional[torch.Tensor],
                   stream: Optional[torch.cuda.Stream] = None) -> None:
         """Packs wave i into its slice of the full-size `buckets` / `checksums` tensors."""

@@ -309,3 +309,28 @@ def test_two_streams_run_independent_plans_concurrently(oracle_mod):
     for k in range(len(b.tensors)):
         assert np.array_equal(tb.host_bytes(k), b.host_bytes(k))
     assert ma.status(s1) == 0 and mb.status(s2) == 0
+
+
+def test_bounded_staging_ring_reproduces_the_stream(oracle_mod):
+    # two staging slots of 2 MiB stand for the recycled transfer channel (paper §8.5): every wave is
+    # packed into a slot, "sent" (copied out), and the slot is reused; the receiver's copy must be the
+    # complete stream, and the checksums the complete list
+    from paper_2412_12636_b200.mover import WaveMover
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    exp_stream, exp_cks = oracle_mod.pack(G.host_tensors(state), cfg.bucket_bytes)
+    wm = WaveMover(state.descs(), cfg.bucket_bytes, 2 << 20)
+    slots = [G.guarded(2 << 20) for _ in range(2)]
+    cks = torch.zeros(wm.n_buckets, dtype=torch.int64, device="cuda")
+    received = torch.empty(wm.total_bytes, dtype=torch.uint8, device="cuda")
+    for i, w in enumerate(wm.waves):
+        whole, slot = slots[i % 2]
+        slot.fill_(0x77)                                   # stale contents of the recycled slot
+        n = wm.pack_wave_into(i, slot, cks)
+        assert n == wm.wave_bytes(i) <= slot.numel()
+        received[w.stream_begin:w.stream_end].copy_(slot[:n])
+        torch.cuda.synchronize()
+        assert G.guards_intact(whole, 2 << 20)
+        assert bool((slot[n:] == 0x77).all())              # nothing written past the wave
+    assert np.array_equal(received.cpu().numpy(), exp_stream)
+    assert np.array_equal(G.u64(cks), exp_cks)
