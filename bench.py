@@ -235,6 +235,8 @@ def run_reference(args) -> None:
     if rank != 0:
         return
     from paper_2412_12636_b200 import layouts
+    if args.workload not in WORKLOADS:
+        raise SystemExit("--impl reference runs on cfg0..cfg3")
     cfg = layouts.role_config(WORKLOADS[args.workload])
     step, sample = oracle_sample_step(cfg, n_layers=1)
     budget_s = 150.0                      # the whole run ends within a few minutes whatever --steps says
@@ -269,10 +271,14 @@ def run_reference(args) -> None:
 class RoleBench:
     """One role on the current GPU with every buffer the step needs."""
 
-    def __init__(self, workload: str):
+    def __init__(self, workload: str, prepared=None):
         from paper_2412_12636_b200 import layouts
         from paper_2412_12636_b200.mover import MultiShardExtractor, RoleMover, ShardExtractor
-        if workload == "cfg4lite":
+        if prepared is not None:      # (RoleState, bucket_bytes, r, D): a wave of a larger role
+            self.state, self.bucket_bytes, self.shard_r, self.shard_D = prepared
+            self.name = self.state.name
+            planes = [self.state.elem_size_indices(4)]
+        elif workload == "cfg4lite":
             self.state = layouts.materialize_adversarial(layouts.adversarial_specs(20_000), "cuda")
             self.name, self.bucket_bytes, self.shard_r, self.shard_D = "adversarial-20000", layouts.ADVERSARIAL_BUCKET, 29, 64
             planes = [self.state.elem_size_indices(4)]
@@ -363,6 +369,65 @@ class RoleBench:
         ops = {n: entry(self.per_op[n], op_ms[n]) for n in ("pack", "checksum", "unpack", "shard")}
         ops["pack+checksum+shard"] = entry(self.per_op["pack"] + self.per_op["shard"], op_ms["pack"] + op_ms["shard"])
         return ops
+
+
+def run_config4_in_waves(args) -> None:
+    """Config 4 as specified (200 000 tensors, about 257 GB of state): more than one GPU holds next
+    to its packed copy, so it is processed in waves of whole buckets (paper_2412_12636_b200/waves.py);
+    throughput = bytes of all waves over the kernel time of all waves."""
+    from paper_2412_12636_b200 import binding, layouts, waves
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    binding.load_library()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    specs = layouts.adversarial_specs(200_000)
+    sizes = [s.nbytes for s in specs]
+    B = layouts.ADVERSARIAL_BUCKET
+    plan = binding.Plan([(0x7F00_0000_0000, n, s.elem_size, s.plane) for n, s in zip(sizes, specs)], B)  # host-only
+    offsets, total, n_buckets = plan.offsets(), plan.total_bytes, plan.n_buckets
+    plan.close()
+    ws = waves.cut_waves(sizes, offsets, total, B, 24 << 30)
+    names = ["pack", "checksum", "unpack", "shard"]
+    sum_ms = {n: 0.0 for n in names}
+    sum_bytes = {n: 0 for n in names}
+    step_ms, step_bytes_total, ok, launches0 = 0.0, 0, True, binding.tm_launch_count()
+    steps = max(2, min(args.steps, 5))
+    for wi, w in enumerate(ws):
+        wave_specs = [specs[p.tensor] for p in w.parts]
+        full = layouts.materialize_adversarial(wave_specs, "cuda", wave=wi)
+        part_specs = [layouts.TensorSpec(s.name, p.nbytes // s.elem_size, s.dtype, s.plane, s.model_index)
+                      for p, s in zip(w.parts, wave_specs)]
+        part_tensors = [t[p.byte_start:p.byte_start + p.nbytes] for p, t in zip(w.parts, full.tensors)]
+        state = layouts.RoleState(f"wave{wi}", part_specs, part_tensors, B, 0, layouts.ADVERSARIAL_D, full.arena)
+        role = RoleBench("cfg4", prepared=(state, B, 29, layouts.ADVERSARIAL_D))
+        for _ in range(2):
+            role.one_step()
+        torch.cuda.synchronize()
+        ms, op_ms = role.timed(steps)
+        ok = ok and role.self_check()
+        step_ms += ms / steps
+        step_bytes_total += role.bytes_per_step
+        for n in names:
+            sum_ms[n] += op_ms[n]
+            sum_bytes[n] += role.per_op[n]
+        del role, state, full, part_tensors
+        torch.cuda.empty_cache()
+    peak, peak_kind = measured_hbm_peak()
+    ops = {n: {"ms": round(sum_ms[n], 4), "GB/s": round(gbs(sum_bytes[n], sum_ms[n]), 1),
+               "frac_of_8TBs_nominal": round(gbs(sum_bytes[n], sum_ms[n]) / NOMINAL_HBM_GBS, 4)} for n in names}
+    line = {"metric": METRIC, "value": round(gbs(step_bytes_total, step_ms), 2), "unit": UNIT, "n_gpus": 1,
+            "steps": steps, "warmup": 2, "ms_per_step": round(step_ms, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u8/u64", "data": "synthetic",
+            "config": {"workload": "cfg4:adversarial-200000", "n_tensors": len(specs), "state_bytes": sum(sizes),
+                       "stream_bytes": total, "n_buckets": n_buckets, "bucket_bytes": B, "waves": len(ws),
+                       "shard": "r=29 of D=64 over each wave's fp32 tensors",
+                       "note": "processed in waves of whole buckets; ms_per_step is the sum over the waves"},
+            "bytes_per_step": step_bytes_total, "ops": ops, "roofline": None, "cpu_baseline": None, "e2e": None,
+            "gpu_launches": binding.tm_launch_count() - launches0, "self_check": "ok" if ok else "MISMATCH",
+            "frac_of_measured_copy": round(gbs(step_bytes_total, step_ms) / peak, 4)}
+    print(json.dumps(line), flush=True)
+    if not ok:
+        raise SystemExit("self-check failed")
 
 
 def run_ours(args) -> None:
@@ -563,13 +628,15 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS) + ["cfg4lite"], default="cfg3")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS) + ["cfg4lite", "cfg4"], default="cfg3")
     ap.add_argument("--also", default="cfg2", help="comma-separated further workloads measured after the main one (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler launch lists)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "cfg4":
+        run_config4_in_waves(args)
     else:
         run_ours(args)
 
