@@ -229,6 +229,23 @@ int tm_checksum(const void* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
  * tm_workspace_status(d_workspace) yields TM_ERR_TIMEOUT.  d_workspace: >= 256 bytes, 256-byte aligned. */
 int tm_selftest_bounded_wait(void* d_workspace, uint64_t limit_ns, void* stream);
 
+/* One piece of a plan's work list, as the kernels see it (for inspection and host-side checks). */
+typedef struct tm_piece {
+  uint64_t tensor;   /* device address of the piece's first tensor byte */
+  uint64_t off;      /* offset of the piece in the packed stream */
+  uint32_t nbytes;   /* tensor bytes in the piece */
+  uint32_t pad;      /* zero bytes that follow it in the stream */
+  uint32_t bucket;   /* bucket the piece lies in */
+  uint32_t word0;    /* index of its first 8-byte word inside that bucket */
+} tm_piece;
+
+/* Copies the plan's work list to host arrays: up to `capacity` pieces into `pieces` and, for every
+ * item, the index of its first piece into `item_first` (n_items + 1 entries, the last one = number
+ * of pieces; `item_capacity` entries available).  Either array may be NULL.  *n_pieces / *n_items
+ * (may be NULL) receive the full counts.  Host only. */
+int tm_plan_pieces(const tm_plan* plan, tm_piece* pieces, uint64_t capacity, uint64_t* n_pieces,
+                   uint32_t* item_first, uint64_t item_capacity, uint64_t* n_items);
+
 /* ---- diagnostics ----------------------------------------------------------------------------- */
 
 const char* tm_strerror(int status);

@@ -24,6 +24,7 @@ SIGNATURES = {
     "tm_plan_create": (_int, [_p, _u64, _u64, _p]),
     "tm_plan_query": (_int, [_p, _p, _p, _p]),
     "tm_plan_offsets": (_int, [_p, _p]),
+    "tm_plan_pieces": (_int, [_p, _p, _u64, _p, _p, _u64, _p]),
     "tm_plan_upload": (_int, [_p, _p, _u64, _p]),
     "tm_plan_status": (_int, [_p, _p, _p]),
     "tm_plan_destroy": (None, [_p]),
@@ -109,6 +110,21 @@ class Plan:
         out = (_u64 * self.n_desc)()
         _check(load_library().tm_plan_offsets(self._h, out), "tm_plan_offsets")
         return list(out)
+
+    def pieces(self):
+        """(pieces, item_first) of the work list as numpy arrays; pieces has fields tensor, off, nbytes,
+        pad, bucket, word0."""
+        import numpy as np
+        L = load_library()
+        np_, ni = _u64(), _u64()
+        _check(L.tm_plan_pieces(self._h, None, 0, ctypes.byref(np_), None, 0, ctypes.byref(ni)), "tm_plan_pieces")
+        dt = np.dtype([("tensor", "<u8"), ("off", "<u8"), ("nbytes", "<u4"), ("pad", "<u4"), ("bucket", "<u4"),
+                       ("word0", "<u4")])
+        pieces = np.zeros(np_.value, dtype=dt)
+        items = np.zeros(ni.value + 1, dtype=np.uint32)
+        _check(L.tm_plan_pieces(self._h, pieces.ctypes.data, pieces.size, None, items.ctypes.data, items.size, None),
+               "tm_plan_pieces")
+        return pieces, items
 
     def upload(self, d_workspace: int, workspace_bytes: int, stream: int) -> None:
         _check(load_library().tm_plan_upload(self._h, d_workspace, workspace_bytes, stream), "tm_plan_upload")

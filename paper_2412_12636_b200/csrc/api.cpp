@@ -163,6 +163,19 @@ int tm_plan_offsets(const tm_plan* plan, uint64_t* offsets) {
   return TM_OK;
 }
 
+int tm_plan_pieces(const tm_plan* plan, tm_piece* pieces, uint64_t capacity, uint64_t* n_pieces,
+                   uint32_t* item_first, uint64_t item_capacity, uint64_t* n_items) {
+  if (plan == nullptr) return TM_ERR_ARG;
+  static_assert(sizeof(tm_piece) == sizeof(tms::Seg), "tm_piece mirrors the internal piece");
+  const uint64_t np = plan->work.segs.size(), ni = plan->work.n_items();
+  if (n_pieces != nullptr) *n_pieces = np;
+  if (n_items != nullptr) *n_items = ni;
+  if (pieces != nullptr) std::memcpy(pieces, plan->work.segs.data(), std::min(np, capacity) * sizeof(tm_piece));
+  if (item_first != nullptr)
+    std::memcpy(item_first, plan->work.item_first.data(), std::min(ni + 1, item_capacity) * sizeof(uint32_t));
+  return TM_OK;
+}
+
 int tm_plan_upload(tm_plan* plan, void* d_workspace, uint64_t workspace_bytes, void* stream) {
   if (plan == nullptr || d_workspace == nullptr) return TM_ERR_ARG;
   if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;

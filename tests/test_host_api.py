@@ -146,3 +146,43 @@ def test_header_is_plain_c_and_library_links_from_c(lib, tmp_path):
     out = subprocess.run([str(exe)], capture_output=True, text=True)
     assert out.returncode == 0, (out.returncode, out.stdout, out.stderr)
     assert "c abi ok, 0 launches" in out.stdout
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_work_list_tiles_the_stream_exactly(lib, oracle_mod, seed):
+    """Planner invariants, checked on the host against the oracle's layout: the pieces cover
+    [0, T) without gap or overlap, stay inside one bucket, carry the right word index and tensor
+    address, and the items partition the pieces within one bucket."""
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(1, 60))
+    log_sizes = rng.uniform(0, 21, n)
+    sizes = [2 * max(1, int(2 ** x) // 2) for x in log_sizes]
+    B = 256 * int(rng.choice([1, 3, 16, 4096, 32768, 1 << 20]))
+    addr, descs = FAKE, []
+    for k, nb in enumerate(sizes):
+        addr += 2 * int(rng.integers(0, 64))
+        descs.append((addr, nb, 2, 0))
+        addr += nb
+    plan = binding.Plan(descs, B)
+    off, T, nbuckets = oracle_mod.layout(sizes, B)
+    pieces, items = plan.pieces()
+    assert items[0] == 0 and items[-1] == pieces.size and np.all(np.diff(items.astype(np.int64)) > 0)
+    pos, k, within = 0, 0, 0          # stream position, current tensor, bytes of it already seen
+    for p in pieces:
+        assert int(p["off"]) == pos and p["nbytes"] > 0 and p["nbytes"] % 2 == 0
+        assert int(p["off"]) == int(off[k]) + within
+        assert int(p["tensor"]) == descs[k][0] + within
+        b = int(p["off"]) // B
+        assert int(p["bucket"]) == b and int(p["word0"]) == (int(p["off"]) - b * B) // 8
+        end = int(p["off"]) + int(p["nbytes"]) + int(p["pad"])
+        assert end <= (b + 1) * B                                   # never crosses a bucket boundary
+        within += int(p["nbytes"])
+        if within == sizes[k]:
+            assert end % 256 == 0 and int(p["pad"]) < 256
+            k, within = k + 1, 0
+        else:
+            assert p["pad"] == 0
+        pos = end
+    assert pos == T and k == n
+    for a, b_ in zip(items[:-1], items[1:]):                        # an item never mixes buckets
+        assert len(set(pieces["bucket"][a:b_].tolist())) == 1
