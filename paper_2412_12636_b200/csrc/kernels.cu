@@ -85,22 +85,21 @@ copy_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
 }
 
 // Stand-alone checksum.  Tile t covers bytes [tile_bytes * (t % tiles_per_bucket), +tile_bytes) of
-// bucket t / tiles_per_bucket.  The input is 16-byte aligned; only the very last vector of the
+// bucket t / tiles_per_bucket (tile_bytes: a multiple of 256, at most 1 GiB).  The input is 16-byte aligned; only the very last vector of the
 // input can be partial.
-constexpr uint32_t kCksumTile = 64 * 1024;
 
 __global__ void __launch_bounds__(kThreads, kMinBlocks)
 checksum_kernel(const uint8_t* __restrict__ bytes, u64 nbytes, u64 bucket_bytes, uint32_t tiles_per_bucket,
-                u64 n_tiles, u64* __restrict__ checksums) {
+                u64 n_tiles, uint32_t tile_bytes, u64* __restrict__ checksums) {
   __shared__ u64 red[kWarps];
   Cksum ck;
   u64 total = 0;
   u64 cur = ~0ull;
   for (u64 t = blockIdx.x; t < n_tiles; t += gridDim.x) {
     const u64 bucket = t / tiles_per_bucket;
-    const u64 in_bucket = (t - bucket * tiles_per_bucket) * (u64)kCksumTile;
+    const u64 in_bucket = (t - bucket * tiles_per_bucket) * (u64)tile_bytes;
     const u64 begin = bucket * bucket_bytes + in_bucket;
-    u64 end = begin + kCksumTile;
+    u64 end = begin + tile_bytes;
     const u64 bucket_end = (bucket + 1) * bucket_bytes;
     if (end > bucket_end) end = bucket_end;
     if (end > nbytes) end = nbytes;
@@ -202,13 +201,14 @@ int launch_copy(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_item
 int launch_checksum(const uint8_t* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
                     unsigned long long* d_checksums, void* stream) {
   const uint64_t n_buckets = (nbytes + bucket_bytes - 1) / bucket_bytes;
-  const uint64_t tpb = (bucket_bytes + kCksumTile - 1) / kCksumTile;
+  const uint32_t tile = (uint32_t)tuning().cksum_tile_bytes;
+  const uint64_t tpb = (bucket_bytes + tile - 1) / tile;
   const uint64_t n_tiles = n_buckets * tpb;
   uint32_t grid = 0;
   int rc = grid_for(n_tiles, &grid);
   if (rc != 0) return rc;
   checksum_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_bytes, nbytes, bucket_bytes, (uint32_t)tpb,
-                                                              n_tiles, d_checksums);
+                                                              n_tiles, tile, d_checksums);
   count_launch();
   return (int)cudaGetLastError();
 }

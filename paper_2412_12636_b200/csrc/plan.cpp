@@ -25,6 +25,8 @@ const Tuning& tuning() {
     if (x.chunk_bytes > (1ull << 30)) x.chunk_bytes = 1ull << 30;
     x.shard_chunk_bytes = align_up(env_u64("TM_SHARD_CHUNK_BYTES", 64 * 1024), 256);
     if (x.shard_chunk_bytes > (1ull << 30)) x.shard_chunk_bytes = 1ull << 30;
+    x.cksum_tile_bytes = align_up(env_u64("TM_CKSUM_TILE_BYTES", 256 * 1024), 256);
+    if (x.cksum_tile_bytes > (1ull << 30)) x.cksum_tile_bytes = 1ull << 30;
     x.small_bytes = env_u64("TM_SMALL_BYTES", 8 * 1024);
     x.group_bytes = env_u64("TM_GROUP_BYTES", 64 * 1024);
     x.group_max = (uint32_t)env_u64("TM_GROUP_MAX", 64);

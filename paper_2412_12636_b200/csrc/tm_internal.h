@@ -52,6 +52,7 @@ struct Tuning {
   uint64_t small_bytes;    // pieces below this share items
   uint64_t group_bytes;    // byte budget of a shared item
   uint32_t group_max;      // piece budget of a shared item
+  uint64_t cksum_tile_bytes;   // tile of the stand-alone checksum kernel; multiple of 256
   uint32_t ctas_per_sm;    // persistent grid = SMs * ctas_per_sm (register-path kernels)
   uint32_t ring_ctas_per_sm;  // same for the bulk-copy ring kernels (96 KiB of shared memory each)
   bool use_ring;           // pack / unpack / shard through the bulk-copy ring kernels
