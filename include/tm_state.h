@@ -146,6 +146,28 @@ int tm_state_unpack(const tm_plan* plan, const void* d_buckets, uint64_t nbytes,
 int tm_state_unpack_verify(const tm_plan* plan, const void* d_buckets, uint64_t nbytes,
                            uint64_t* d_checksums, void* stream);
 
+/* Pack that also emits shards (the leaver, or a stayer holding a replica, hands a joiner both the
+ * packed role and the slice of the optimizer state its data-parallel rank owns — §7 "State
+ * Synchronization" — reading every tensor once).
+ *
+ * tm_plan_attach_shards prepares it: planes are runs of the plan's own descriptors — plane p is
+ * descriptors [plane_first_desc[p], + plane_n_desc[p]), runs ascending and disjoint, one elem_size
+ * per plane — and each is sliced with the same r and D exactly as by tm_shard_extract, into
+ * d_outs[p] (capacity out_capacities[p]).  The merged work list (every tensor's pack pieces followed
+ * by the emit pieces that read the same tensor, so that the second read is served by the L2) is
+ * uploaded once to d_workspace on `stream`.  With d_workspace == NULL nothing is uploaded and only
+ * *workspace_needed (may be NULL otherwise) and out_elems (n_planes entries, may be NULL) are filled.
+ * The outputs must not overlap the tensors, one another, or the packed buffer used later.
+ *
+ * tm_state_pack_emit then does what tm_state_pack does (same arguments, same results) and fills the
+ * attached shard outputs in the same launch. */
+int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const uint64_t* plane_n_desc,
+                          uint32_t n_planes, uint32_t r, uint32_t D, void* const* d_outs,
+                          const uint64_t* out_capacities, uint64_t* out_elems, void* d_workspace,
+                          uint64_t workspace_bytes, uint64_t* workspace_needed, void* stream);
+int tm_state_pack_emit(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint64_t* d_checksums,
+                       void* stream);
+
 /* Host helper: floor shard bounds lo = floor(r*N/D), hi = floor((r+1)*N/D) in 128-bit arithmetic. */
 int tm_shard_bounds(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
 

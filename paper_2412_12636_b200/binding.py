@@ -31,6 +31,8 @@ SIGNATURES = {
     "tm_state_pack": (_int, [_p, _p, _u64, _p, _p]),
     "tm_state_unpack": (_int, [_p, _p, _u64, _p]),
     "tm_state_unpack_verify": (_int, [_p, _p, _u64, _p, _p]),
+    "tm_plan_attach_shards": (_int, [_p, _p, _p, _u32, _u32, _u32, _p, _p, _p, _p, _u64, _p, _p]),
+    "tm_state_pack_emit": (_int, [_p, _p, _u64, _p, _p]),
     "tm_shard_bounds": (_int, [_u64, _u32, _u32, _p, _p]),
     "tm_shard_workspace": (_int, [_p, _u64, _u32, _u32, _p]),
     "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
@@ -161,6 +163,27 @@ def tm_state_unpack(plan: Plan, d_buckets: int, nbytes: int, stream: int) -> Non
 def tm_state_unpack_verify(plan: Plan, d_buckets: int, nbytes: int, d_checksums: int, stream: int) -> None:
     _check(load_library().tm_state_unpack_verify(plan.handle, d_buckets, nbytes, d_checksums, stream),
            "tm_state_unpack_verify")
+
+
+def tm_plan_attach_shards(plan: Plan, planes: Sequence[Tuple[int, int]], r: int, D: int,
+                          d_outs: Optional[Sequence[int]], out_capacities: Optional[Sequence[int]],
+                          d_workspace: Optional[int], workspace_bytes: int, stream: int) -> Tuple[List[int], int]:
+    """`planes` = (first descriptor, count) per plane.  Returns (elements per shard, workspace bytes
+    needed); with d_workspace None nothing is uploaded (size query)."""
+    n = len(planes)
+    first = (_u64 * n)(*[p[0] for p in planes])
+    count = (_u64 * n)(*[p[1] for p in planes])
+    outs = (_p * n)(*d_outs) if d_outs is not None else None
+    caps = (_u64 * n)(*out_capacities) if out_capacities is not None else None
+    got, need = (_u64 * n)(), _u64()
+    _check(load_library().tm_plan_attach_shards(plan.handle, first, count, n, r, D, outs, caps, got, d_workspace,
+                                                workspace_bytes, ctypes.byref(need), stream), "tm_plan_attach_shards")
+    return list(got), need.value
+
+
+def tm_state_pack_emit(plan: Plan, d_buckets: int, capacity: int, d_checksums: Optional[int], stream: int) -> None:
+    _check(load_library().tm_state_pack_emit(plan.handle, d_buckets, capacity, d_checksums, stream),
+           "tm_state_pack_emit")
 
 
 def tm_shard_bounds(n_elems: int, r: int, D: int) -> Tuple[int, int]:

@@ -20,7 +20,7 @@ void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64
                        uint64_t d_out, tms::WorkList* wl);
 int tm_targets_disjoint(const tm_plan* p);
 void tm_shard_append(tms::WorkListBuilder* builder, const tm_desc* descs, uint64_t n_desc, uint32_t e,
-                     uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base);
+                     uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base, uint32_t bucket_tag);
 
 namespace {
 
@@ -187,9 +187,19 @@ int tm_plan_upload(tm_plan* plan, void* d_workspace, uint64_t workspace_bytes, v
 }
 
 int tm_plan_status(const tm_plan* plan, void* stream, int* device_status) {
-  if (plan == nullptr) return TM_ERR_ARG;
-  if (plan->d_workspace == nullptr) return TM_ERR_STATE;
-  return read_status(plan->d_workspace, (cudaStream_t)stream, device_status);
+  if (plan == nullptr || device_status == nullptr) return TM_ERR_ARG;
+  if (plan->d_workspace == nullptr && plan->d_emit_workspace == nullptr) return TM_ERR_STATE;
+  int a = 0, b = 0;
+  if (plan->d_workspace != nullptr) {
+    int rc = read_status(plan->d_workspace, (cudaStream_t)stream, &a);
+    if (rc != TM_OK) return rc;
+  }
+  if (plan->d_emit_workspace != nullptr) {
+    int rc = read_status(plan->d_emit_workspace, (cudaStream_t)stream, &b);
+    if (rc != TM_OK) return rc;
+  }
+  *device_status = (a != 0) ? a : b;
+  return TM_OK;
 }
 
 void tm_plan_destroy(tm_plan* plan) { delete plan; }
@@ -251,6 +261,116 @@ int tm_state_unpack_verify(const tm_plan* plan, const void* d_buckets, uint64_t 
                                          (const uint32_t*)(ws + plan->ws_layout.items_off),
                                          (uint32_t)plan->work.n_items(), (uint8_t*)const_cast<void*>(d_buckets),
                                          (unsigned long long*)d_checksums, (int*)plan->d_workspace, stream);
+  return e == 0 ? TM_OK : cuda_fail(e);
+}
+
+int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const uint64_t* plane_n_desc,
+                          uint32_t n_planes, uint32_t r, uint32_t D, void* const* d_outs,
+                          const uint64_t* out_capacities, uint64_t* out_elems, void* d_workspace,
+                          uint64_t workspace_bytes, uint64_t* workspace_needed, void* stream) {
+  if (plan == nullptr || plane_first_desc == nullptr || plane_n_desc == nullptr || n_planes == 0)
+    return TM_ERR_ARG;
+  if (D == 0 || r >= D) return TM_ERR_RANK;
+  const uint64_t n_desc = plan->descs.size();
+  struct PlaneInfo { uint64_t first, n; uint32_t e; uint64_t lo, hi; };
+  std::vector<PlaneInfo> planes(n_planes);
+  uint64_t prev_end = 0;
+  for (uint32_t p = 0; p < n_planes; ++p) {
+    PlaneInfo& pi = planes[p];
+    pi.first = plane_first_desc[p];
+    pi.n = plane_n_desc[p];
+    if (pi.n == 0 || pi.first < prev_end || pi.first + pi.n > n_desc) return TM_ERR_ARG;   // ascending, disjoint
+    prev_end = pi.first + pi.n;
+    uint64_t n_elems = 0;
+    int rc = tm_shard_validate(plan->descs.data() + pi.first, pi.n, r, D, &pi.e, &n_elems);
+    if (rc != TM_OK) return rc;
+    rc = tm_bounds_u128(n_elems, r, D, &pi.lo, &pi.hi);
+    if (rc != TM_OK) return rc;
+    if (out_elems != nullptr) out_elems[p] = pi.hi - pi.lo;
+  }
+  const bool dry = (d_workspace == nullptr);
+  uint64_t base = ~0ull;
+  std::vector<std::pair<uint64_t, uint64_t>> outs;
+  if (!dry) {
+    if (d_outs == nullptr || out_capacities == nullptr) return TM_ERR_ARG;
+    if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+    for (uint32_t p = 0; p < n_planes; ++p) {
+      const uint64_t bytes = (planes[p].hi - planes[p].lo) * planes[p].e;
+      if (bytes == 0) continue;
+      if (d_outs[p] == nullptr) return TM_ERR_ARG;
+      if (((uintptr_t)d_outs[p] & 1) != 0) return TM_ERR_ALIGN;
+      if (out_capacities[p] < bytes) return TM_ERR_CAPACITY;
+      const uint64_t o = (uint64_t)(uintptr_t)d_outs[p];
+      for (const tm_desc& d : plan->descs)
+        if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, o, bytes)) return TM_ERR_OVERLAP;
+      for (const auto& q : outs)
+        if (ranges_overlap(o, bytes, q.first, q.second)) return TM_ERR_OVERLAP;
+      outs.emplace_back(o, bytes);
+      base = std::min(base, o);
+    }
+  }
+  if (base == ~0ull) base = 0;
+  // one pass over the descriptors: the pack pieces of tensor k, then the emit pieces that read tensor k
+  tms::WorkList wl;
+  tms::WorkListBuilder builder(&wl);
+  size_t cursor = 0;            // next pack piece of the plan
+  uint32_t p = 0;               // current plane
+  uint64_t start = 0;           // element index, inside plane p, of tensor k's first element
+  for (uint64_t k = 0; k < n_desc; ++k) {
+    uint64_t seen = 0;
+    while (seen < plan->descs[k].nbytes) {
+      const tms::Seg& s = plan->work.segs[cursor++];
+      builder.add(s);
+      seen += s.nbytes;
+    }
+    while (p < n_planes && k >= planes[p].first + planes[p].n) { ++p; start = 0; }
+    if (p < n_planes && k >= planes[p].first) {
+      const PlaneInfo& pi = planes[p];
+      const uint64_t count = plan->descs[k].nbytes / pi.e;
+      const uint64_t a = std::max(pi.lo, start), b = std::min(pi.hi, start + count);
+      if (a < b) {
+        const uint64_t out = dry ? (uint64_t)256 * (a - pi.lo) : (uint64_t)(uintptr_t)d_outs[p] + (a - pi.lo) * pi.e;
+        tm_shard_append(&builder, &plan->descs[k], 1, pi.e, a - start, b - start, out, dry ? 0 : base, 0xffffffffu);
+      }
+      start += count;
+    }
+  }
+  builder.finish();
+  const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size() + 2 * n_desc + 8, wl.n_items() + 2 * n_desc + 8);
+  if (workspace_needed != nullptr) *workspace_needed = l.total;
+  if (dry) return TM_OK;
+  const tms::WorkspaceLayout exact = tms::workspace_layout(wl.segs.size(), wl.n_items());
+  if (workspace_bytes < exact.total) return TM_ERR_CAPACITY;
+  int rc = upload_worklist(wl, exact, (uint8_t*)d_workspace, (cudaStream_t)stream);
+  if (rc != TM_OK) return rc;
+  plan->emit_work = std::move(wl);
+  plan->emit_layout = exact;
+  plan->d_emit_workspace = (uint8_t*)d_workspace;
+  plan->emit_base = base;
+  plan->emit_outs = std::move(outs);
+  return TM_OK;
+}
+
+int tm_state_pack_emit(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint64_t* d_checksums,
+                       void* stream) {
+  if (plan == nullptr || d_buckets == nullptr) return TM_ERR_ARG;
+  if (plan->d_emit_workspace == nullptr) return TM_ERR_STATE;
+  if (((uintptr_t)d_buckets & 255) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
+  if (capacity < plan->total_bytes) return TM_ERR_CAPACITY;
+  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
+  for (const tm_desc& d : plan->descs)
+    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
+  for (const auto& o : plan->emit_outs)
+    if (ranges_overlap(o.first, o.second, base, plan->total_bytes)) return TM_ERR_OVERLAP;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (d_checksums != nullptr)
+    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), st));
+  const uint8_t* ws = plan->d_emit_workspace;
+  int e = tms::launch_pack_emit_ring((const tms::Seg*)(ws + plan->emit_layout.segs_off),
+                                     (const uint32_t*)(ws + plan->emit_layout.items_off),
+                                     (uint32_t)plan->emit_work.n_items(), (uint8_t*)d_buckets,
+                                     (unsigned long long*)d_checksums, (uint8_t*)(uintptr_t)plan->emit_base,
+                                     (int*)plan->d_emit_workspace, stream);
   return e == 0 ? TM_OK : cuda_fail(e);
 }
 
@@ -366,7 +486,7 @@ int tm_shard_extract_planes(const tm_desc* descs, const uint64_t* plane_n_desc, 
   for (uint32_t p = 0; p < n_planes; ++p)
     if (planes[p].hi != planes[p].lo)
       tm_shard_append(&builder, planes[p].d, planes[p].n, planes[p].e, planes[p].lo, planes[p].hi,
-                      (uint64_t)(uintptr_t)d_outs[p], base);
+                      (uint64_t)(uintptr_t)d_outs[p], base, 0);
   builder.finish();
   const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
   if (workspace_bytes < l.total) return TM_ERR_CAPACITY;

@@ -177,7 +177,7 @@ int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_
 // d_out; piece offsets are relative to `flat_base` (<= d_out).  Pieces after the first of each
 // tensor start on a 256-byte boundary of the output.
 void tm_shard_append(tms::WorkListBuilder* builder, const tm_desc* descs, uint64_t n_desc, uint32_t e,
-                     uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base) {
+                     uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base, uint32_t bucket_tag) {
   const uint64_t chunk = tms::tuning().shard_chunk_bytes;
   uint64_t start = 0;  // element index of the tensor's first element in the flat plane
   for (uint64_t k = 0; k < n_desc && start < hi; ++k) {
@@ -198,7 +198,7 @@ void tm_shard_append(tms::WorkListBuilder* builder, const tm_desc* descs, uint64
         s.off = (d_out - flat_base) + out;
         s.nbytes = (uint32_t)len;
         s.pad = 0;
-        s.bucket = 0;
+        s.bucket = bucket_tag;
         s.word0 = 0;
         builder->add(s);
         tensor += len;
@@ -214,7 +214,7 @@ void tm_shard_append(tms::WorkListBuilder* builder, const tm_desc* descs, uint64
 void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
                        uint64_t d_out, tms::WorkList* wl) {
   tms::WorkListBuilder builder(wl);
-  tm_shard_append(&builder, descs, n_desc, e, lo, hi, d_out, d_out);
+  tm_shard_append(&builder, descs, n_desc, e, lo, hi, d_out, d_out, 0);
   builder.finish();
 }
 

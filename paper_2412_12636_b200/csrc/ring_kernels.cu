@@ -35,6 +35,7 @@ constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kRingThreads = kConsThreads + 64;     // + one producer warp + one store warp
 constexpr uint32_t kBulkMinVectors = 128;           // pieces below 2 KiB are not worth a stage
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr uint32_t kEmitBucket = 0xffffffffu;       // marks an emit piece in a pack-and-emit list
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
@@ -154,10 +155,14 @@ __device__ __forceinline__ void consumer_flush(u64 value, u64* target) {
 // given by TO_TENSORS (PACK implies TO_TENSORS == false).  VERIFY (with TO_TENSORS): the unpack also
 // accumulates the per-bucket checksums of the stream it reads — data and padding bytes as they
 // arrived — so that a receiver checks and scatters in one pass over the buckets.
-template <bool PACK, bool TO_TENSORS, bool VERIFY>
+// EMIT (with PACK): the list also holds "emit" pieces, marked by bucket == kEmitBucket, which are
+// plain copies tensor -> flat2 (a shard output); they sit next to the pack pieces that read the same
+// tensor bytes, so their source is served from the L2 rather than read from DRAM a second time.
+template <bool PACK, bool TO_TENSORS, bool VERIFY, bool EMIT>
 __global__ void __launch_bounds__(kRingThreads, 1)
 ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
-            uint8_t* __restrict__ flat, u64* __restrict__ checksums, int* __restrict__ status) {
+            uint8_t* __restrict__ flat, u64* __restrict__ checksums, int* __restrict__ status,
+            uint8_t* __restrict__ flat2) {
   extern __shared__ __align__(128) uint8_t ring[];
   __shared__ RingShared sh;
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -182,7 +187,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       if (item_first[item + 1] - first != 1) continue;
       const Seg s = segs[first];
       BulkPlan p;
-      if (!plan_bulk<TO_TENSORS>(s, flat, p)) continue;
+      if (!plan_bulk<TO_TENSORS>(s, (EMIT && s.bucket == kEmitBucket) ? flat2 : flat, p)) continue;
       const uint32_t extra = p.a != 0 ? 1u : 0u;
       for (uint32_t t = 0; t < p.ntiles; ++t) {
         if (!mbar_wait(&sh.empty[stage], phase ^ 1u, abort_flag)) {
@@ -224,7 +229,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       if (item_first[item + 1] - first != 1) continue;
       const Seg s = segs[first];
       BulkPlan p;
-      if (!plan_bulk<TO_TENSORS>(s, flat, p)) continue;
+      if (!plan_bulk<TO_TENSORS>(s, (EMIT && s.bucket == kEmitBucket) ? flat2 : flat, p)) continue;
       for (uint32_t t = 0; t < p.ntiles; ++t) {
         if (!mbar_wait(&sh.full[stage], phase, abort_flag)) {
           raise_timeout(status, &sh);
@@ -267,7 +272,10 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
   bool ok = true;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t first = item_first[item], last = item_first[item + 1];
-    if (PACK || VERIFY) {
+    const bool emit_item = EMIT && segs[first].bucket == kEmitBucket;   // uniform over the block
+    const bool packing = PACK && !emit_item;
+    uint8_t* const base = emit_item ? flat2 : flat;
+    if ((PACK || VERIFY) && !emit_item) {
       const uint32_t bucket = segs[first].bucket;
       if (bucket != cur) {   // uniform over the consumers
         if (cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur);
@@ -281,19 +289,19 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
     bool bulk = false;
     if (single) {
       s0 = segs[first];
-      bulk = plan_bulk<TO_TENSORS>(s0, flat, p);
+      bulk = plan_bulk<TO_TENSORS>(s0, base, p);
     }
     if (!bulk) {
       if (!ok) continue;
       const uint32_t g = single ? c : lane, G = single ? (uint32_t)kConsThreads : 32u;
       for (uint32_t i = first + (single ? 0u : warp); i < last; i += (single ? 1u : (uint32_t)kConsWarps)) {
         const Seg s = segs[i];
-        if (PACK) {
+        if (packing) {
           pack_piece(s, flat, g, G, ck);
           total += ck.finish(s.word0);
         } else {
           uint8_t* t = reinterpret_cast<uint8_t*>(s.tensor);
-          uint8_t* f = flat + s.off;
+          uint8_t* f = base + s.off;
           copy_piece(TO_TENSORS ? t : f, TO_TENSORS ? f : t, s.nbytes, g, G);
           if (VERIFY) {   // the piece's span of the stream, padding included, in aligned vectors
             const uint32_t nvec = (s.nbytes + s.pad) >> 4;
@@ -323,7 +331,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       uint8_t* d = p.dst + (size_t)vbase * 16u;
       // VERIFY: the stream piece starts 256-byte aligned, so stage vector v is stream vector vbase + v
       if (p.straight) {
-        if (PACK || VERIFY) {   // the store thread moves the data; only the checksum is left to do
+        if (packing || VERIFY) {   // the store thread moves the data; only the checksum is left to do
 #pragma unroll 4
           for (uint32_t v = c; v < cnt; v += kConsThreads) ck.add(sp[v], vbase + v);
         }
@@ -333,7 +341,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
           const uint4 lo = sp[v];
           const uint4 x = shift_pair(lo, sp[v + 1], ws, bs);
           st16(d + (size_t)v * 16u, x);
-          if (PACK) ck.add(x, vbase + v);
+          if (packing) ck.add(x, vbase + v);
           if (VERIFY) ck.add(lo, vbase + v);
         }
       }
@@ -342,7 +350,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
     }
     if (!ok) continue;
-    if (PACK) {
+    if (packing) {
       // the vector with the tensor's last (n mod 16) bytes, then whole vectors of zero padding
       const uint32_t nvec = (s0.nbytes + s0.pad) >> 4;
       for (uint32_t v = p.nfull + c; v < nvec; v += kConsThreads) {
@@ -396,7 +404,7 @@ int launch_wait_selftest(int* d_status, unsigned long long limit_ns, void* strea
 
 template <typename K>
 static int launch_ring(K kernel, const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
-                       unsigned long long* d_checksums, int* d_status, void* stream) {
+                       unsigned long long* d_checksums, int* d_status, void* stream, uint8_t* d_flat2 = nullptr) {
   int sms = 0;
   int rc = device_sm_count(&sms);
   if (rc != 0) return rc;
@@ -407,28 +415,34 @@ static int launch_ring(K kernel, const Seg* d_segs, const uint32_t* d_item_first
   if (grid > n_items) grid = n_items;
   if (grid == 0) grid = 1;
   kernel<<<(uint32_t)grid, kRingThreads, smem, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat,
-                                                                    d_checksums, d_status);
+                                                                    d_checksums, d_status, d_flat2);
   count_launch();
   return (int)cudaGetLastError();
 }
 
 int launch_pack_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
                      unsigned long long* d_checksums, int* d_status, void* stream) {
-  return launch_ring(ring_kernel<true, false, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
+  return launch_ring(ring_kernel<true, false, false, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
                      stream);
 }
 
 int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
                      bool to_tensors, int* d_status, void* stream) {
   if (to_tensors)
-    return launch_ring(ring_kernel<false, true, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
-  return launch_ring(ring_kernel<false, false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
+    return launch_ring(ring_kernel<false, true, false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
+  return launch_ring(ring_kernel<false, false, false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
 }
 
 int launch_unpack_verify_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
                               unsigned long long* d_checksums, int* d_status, void* stream) {
-  return launch_ring(ring_kernel<false, true, true>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
+  return launch_ring(ring_kernel<false, true, true, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
                      stream);
+}
+
+int launch_pack_emit_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
+                          unsigned long long* d_checksums, uint8_t* d_emit_base, int* d_status, void* stream) {
+  return launch_ring(ring_kernel<true, false, false, true>, d_segs, d_item_first, n_items, d_stream, d_checksums,
+                     d_status, stream, d_emit_base);
 }
 
 }  // namespace tms

@@ -3,6 +3,7 @@
 #define TM_INTERNAL_H
 
 #include <cstdint>
+#include <utility>
 #include <vector>
 
 #include "tm_state.h"
@@ -83,6 +84,8 @@ int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n
                      bool to_tensors, int* d_status, void* stream);
 int launch_unpack_verify_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
                               unsigned long long* d_checksums, int* d_status, void* stream);
+int launch_pack_emit_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
+                          unsigned long long* d_checksums, uint8_t* d_emit_base, int* d_status, void* stream);
 int launch_wait_selftest(int* d_status, unsigned long long limit_ns, void* stream);
 int launch_checksum(const uint8_t* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
                     unsigned long long* d_checksums, void* stream);
@@ -101,6 +104,12 @@ struct tm_plan {
   tms::WorkspaceLayout ws_layout{};
   // set by tm_plan_upload
   uint8_t* d_workspace = nullptr;
+  // set by tm_plan_attach_shards: pack pieces interleaved with the emit pieces of the attached shards
+  tms::WorkList emit_work;
+  tms::WorkspaceLayout emit_layout{};
+  uint8_t* d_emit_workspace = nullptr;
+  uint64_t emit_base = 0;                      // lowest shard output address; emit offsets are relative to it
+  std::vector<std::pair<uint64_t, uint64_t>> emit_outs;   // (address, bytes) of every non-empty shard output
   // lazily computed: 0 unknown, 1 targets disjoint, -1 targets overlap
   mutable int targets_disjoint = 0;
 };

@@ -20,6 +20,7 @@ class RoleMover:
                  stream: Optional[torch.cuda.Stream] = None):
         self.device = torch.device(device)
         self.plan = binding.Plan(descs, bucket_bytes)
+        self._elem_sizes = [d[2] for d in descs]
         self.total_bytes = self.plan.total_bytes
         self.n_buckets = self.plan.n_buckets
         self.bucket_bytes = bucket_bytes
@@ -37,6 +38,26 @@ class RoleMover:
              stream: Optional[torch.cuda.Stream] = None) -> None:
         binding.tm_state_pack(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
                               None if checksums is None else checksums.data_ptr(), _stream_handle(stream))
+
+    def attach_shards(self, planes: Sequence[Tuple[int, int]], r: int, D: int,
+                      stream: Optional[torch.cuda.Stream] = None):
+        """Prepares pack_emit: `planes` = (first descriptor, count) runs of this role's descriptors.
+        Allocates and returns the shard output buffers (one uint8 tensor per plane)."""
+        elems, need = binding.tm_plan_attach_shards(self.plan, planes, r, D, None, None, None, 0, 0)
+        sizes = []
+        for (first, count), n in zip(planes, elems):
+            sizes.append(n * self._elem_sizes[first])
+        self.emit_outs = [torch.empty(max(n, 1), dtype=torch.uint8, device=self.device)[:n] for n in sizes]
+        self.emit_workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        binding.tm_plan_attach_shards(self.plan, planes, r, D, [o.data_ptr() for o in self.emit_outs], sizes,
+                                      self.emit_workspace.data_ptr(), need, _stream_handle(stream))
+        return self.emit_outs
+
+    def pack_emit(self, buckets: torch.Tensor, checksums: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> None:
+        """pack + the attached shards in one launch."""
+        binding.tm_state_pack_emit(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
+                                   None if checksums is None else checksums.data_ptr(), _stream_handle(stream))
 
     def unpack(self, buckets: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
         binding.tm_state_unpack(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),

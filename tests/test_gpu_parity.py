@@ -334,3 +334,51 @@ def test_bounded_staging_ring_reproduces_the_stream(oracle_mod):
         assert bool((slot[n:] == 0x77).all())              # nothing written past the wave
     assert np.array_equal(received.cpu().numpy(), exp_stream)
     assert np.array_equal(G.u64(cks), exp_cks)
+
+
+def test_pack_emit_gives_the_stream_and_the_shards_in_one_launch(oracle_mod):
+    cases = []
+    cfg = layouts.role_config(0)
+    st0 = layouts.materialize(cfg, "cuda")
+    P = len(cfg.model)
+    cases.append((st0, [(P, P), (2 * P, P), (3 * P, P)], 1, 2, cfg.bucket_bytes))
+    cases.append((st0, [(P, P), (3 * P, P)], 2, 3, 256 * 1024))                    # mid-tensor bounds, two planes
+    specs = sorted(layouts.adversarial_specs(500, max_log2=17), key=lambda s: s.elem_size)   # runs per element size
+    adv = layouts.materialize_adversarial(specs, "cuda", seed=9)
+    runs, k = [], 0
+    for e in (2, 4, 8):
+        n = sum(1 for s in specs if s.elem_size == e)
+        runs.append((k, n))
+        k += n
+    cases.append((adv, runs, 5, 7, 1 << 20))
+    cases.append((adv, runs[1:2], 63, 64, 1 << 20))
+    for state, planes, r, D, B in cases:
+        host = G.host_tensors(state)
+        exp_stream, exp_cks = oracle_mod.pack(host, B)
+        mover = RoleMover(state.descs(), B)
+        outs = mover.attach_shards(planes, r, D)
+        whole, buckets = G.guarded(mover.total_bytes)
+        cks = mover.alloc_checksums()
+        launches = binding.tm_launch_count()
+        mover.pack_emit(buckets, cks)
+        torch.cuda.synchronize()
+        assert binding.tm_launch_count() == launches + 1
+        assert mover.status() == 0 and G.guards_intact(whole, mover.total_bytes)
+        assert np.array_equal(buckets.cpu().numpy(), exp_stream)
+        assert np.array_equal(G.u64(cks), exp_cks)
+        for (first, count), out in zip(planes, outs):
+            e = state.specs[first].elem_size
+            sub = host[first:first + count]
+            expect = oracle_mod.shard(sub, [h.size for h in sub], e, r, D)
+            assert np.array_equal(out.cpu().numpy(), expect), (first, count, r, D)
+    # argument checks: overlapping or descending planes, unattached plan
+    plain = RoleMover(st0.descs(), 1 << 20)
+    with pytest.raises(binding.TmError) as ex:
+        binding.tm_state_pack_emit(plain.plan, 1 << 40, 1 << 40, None, 0)
+    assert ex.value.status == binding.TM_ERR_STATE
+    with pytest.raises(binding.TmError) as ex:
+        binding.tm_plan_attach_shards(plain.plan, [(2 * P, P), (P, P)], 0, 2, None, None, None, 0, 0)
+    assert ex.value.status == binding.TM_ERR_ARG
+    with pytest.raises(binding.TmError) as ex:
+        binding.tm_plan_attach_shards(plain.plan, [(0, 2 * P)], 0, 2, None, None, None, 0, 0)   # bf16 + fp32 in one plane
+    assert ex.value.status == binding.TM_ERR_DTYPE
