@@ -354,6 +354,26 @@ class RoleBench:
         return {"ms": round(ms, 4), "GB/s": round(gbs(nbytes, ms), 1),
                 "checksums_match": bool(torch.equal(got, self.cks_fused))}
 
+    def time_pack_emit(self, steps: int):
+        """tm_state_pack_emit (pack + the three fp32 shards in one launch) against pack, then shard."""
+        P = len(self.state.specs) // 4
+        if self.state.arena is not None or any(s.plane != k // P for k, s in enumerate(self.state.specs)):
+            return None                       # planes are not contiguous descriptor runs in this layout
+        outs = self.mover.attach_shards([(P, P), (2 * P, P), (3 * P, P)], self.shard_r, self.shard_D)
+        cks = self.mover.alloc_checksums()
+        for _ in range(2):
+            self.mover.pack_emit(self.buckets, cks)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(self.stream)
+        for _ in range(steps):
+            self.mover.pack_emit(self.buckets, cks)
+        b.record(self.stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / steps
+        nbytes = self.per_op["pack"] + self.per_op["shard"]
+        same = bool(torch.equal(cks, self.cks_fused)) and all(torch.equal(o, m) for o, m in zip(outs, self.multi_outs))
+        return {"ms": round(ms, 4), "GB/s": round(gbs(nbytes, ms), 1), "outputs_match": same}
+
     def self_check(self) -> bool:
         from paper_2412_12636_b200 import layouts
         ok = self.mover.status() == 0 and self.unmover.status() == 0
@@ -470,6 +490,8 @@ def run_ours(args) -> None:
     ok = role.self_check()
     fused_receive = role.time_fused_receive(max(3, args.steps // 2)) if rank == 0 else None
     ok = ok and (fused_receive is None or fused_receive["checksums_match"])
+    fused_send = role.time_pack_emit(max(3, args.steps // 2)) if rank == 0 else None
+    ok = ok and (fused_send is None or fused_send["outputs_match"])
 
     total_ms, total_bytes = aggregate_over_ranks(elapsed_ms, role.bytes_per_step * args.steps)
     peak, peak_kind = measured_hbm_peak()
@@ -529,6 +551,9 @@ def run_ours(args) -> None:
         "fused_receive": fused_receive and dict(fused_receive, note="tm_state_unpack_verify: unpack + checksum of the received "
                                                 "buckets in one pass; not part of the timed step",
                                                 separate_ms=round(ops["checksum"]["ms"] + ops["unpack"]["ms"], 4)),
+        "fused_send": fused_send and dict(fused_send, note="tm_state_pack_emit: pack + fused checksum + the three shards in one "
+                                          "launch; not part of the timed step",
+                                          separate_ms=round(ops["pack"]["ms"] + ops["shard"]["ms"], 4)),
         "also": also,
     }
     print(json.dumps(line), flush=True)
