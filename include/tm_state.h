@@ -52,6 +52,8 @@
  *     Functions return TM_OK (0) or a negative tm_status.  On error nothing has
  *     been enqueued.  There is no CPU fallback: without a usable CUDA device
  *     the operations return TM_ERR_CUDA.
+ *   - Calls are thread-safe with respect to one another, but one tm_plan must not
+ *     be used by two threads at the same time.
  *   - Tensor addresses need only 2-byte alignment.  To serve such tensors at
  *     full speed the kernels read whole 16-byte-aligned lines: a line that
  *     holds at least one byte of a tensor may be read in full (it lies in the
