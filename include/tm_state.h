@@ -98,7 +98,7 @@ typedef struct tm_plan tm_plan;  /* opaque */
  * descriptors and cuts it into the device work list.  Host only: no CUDA call is made.
  * `descs` is copied; it may be freed after the call.  *out receives a plan to be released with
  * tm_plan_destroy.  Errors: TM_ERR_ARG (NULL, n_desc == 0, nbytes == 0, nbytes % elem_size != 0,
- * bucket_bytes == 0 or > 2^35), TM_ERR_DTYPE, TM_ERR_ALIGN (odd ptr, bucket_bytes % 256 != 0). */
+ * bucket_bytes == 0 or > 2^35, nbytes > 2^46, n_desc > 2^24), TM_ERR_DTYPE, TM_ERR_ALIGN (odd ptr, bucket_bytes % 256 != 0). */
 int tm_plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_plan** out);
 
 /* Any of the three outputs may be NULL.  total_bytes = T, n_buckets = ceil(T/B),

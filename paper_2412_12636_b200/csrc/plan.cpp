@@ -101,8 +101,10 @@ int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bu
     const tm_desc& d = descs[k];
     if (d.elem_size != 2 && d.elem_size != 4 && d.elem_size != 8) return TM_ERR_DTYPE;
     if (d.ptr == nullptr || d.nbytes == 0 || d.nbytes % d.elem_size != 0) return TM_ERR_ARG;
+    if (d.nbytes > (1ull << 46)) return TM_ERR_ARG;   // keeps every offset far from 64-bit wrap-around
     if (((uintptr_t)d.ptr & 1) != 0) return TM_ERR_ALIGN;
   }
+  if (n_desc > (1ull << 24)) return TM_ERR_ARG;
   p->descs.assign(descs, descs + n_desc);
   p->bucket_bytes = bucket_bytes;
   p->offsets.resize(n_desc);

@@ -73,6 +73,7 @@ def test_plan_rejects_bad_arguments(lib):
         ([(FAKE, 6, 3, 0)], 256, binding.TM_ERR_DTYPE),
         ([(0, 4, 2, 0)], 256, binding.TM_ERR_ARG),
         ([], 256, binding.TM_ERR_ARG),
+        ([(FAKE, (1 << 46) + 2, 2, 0)], 256, binding.TM_ERR_ARG),   # absurd size: refused, no overflow
     ]
     for descs, B, code in cases:
         with pytest.raises(binding.TmError) as e:
