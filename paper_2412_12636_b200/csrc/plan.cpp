@@ -158,7 +158,7 @@ int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint6
 // Validates a shard plane and returns its element size and element count.
 int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_t D,
                       uint32_t* elem_size, uint64_t* n_elems) {
-  if (descs == nullptr || n_desc == 0) return TM_ERR_ARG;
+  if (descs == nullptr || n_desc == 0 || n_desc > (1ull << 24)) return TM_ERR_ARG;
   if (D == 0 || r >= D) return TM_ERR_RANK;
   const uint32_t e = descs[0].elem_size;
   if (e != 2 && e != 4 && e != 8) return TM_ERR_DTYPE;
@@ -166,7 +166,7 @@ int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_
   for (uint64_t k = 0; k < n_desc; ++k) {
     const tm_desc& d = descs[k];
     if (d.elem_size != e) return TM_ERR_DTYPE;
-    if (d.ptr == nullptr || d.nbytes == 0 || d.nbytes % e != 0) return TM_ERR_ARG;
+    if (d.ptr == nullptr || d.nbytes == 0 || d.nbytes % e != 0 || d.nbytes > (1ull << 46)) return TM_ERR_ARG;
     if (((uintptr_t)d.ptr & 1) != 0) return TM_ERR_ALIGN;
     total += d.nbytes / e;
   }
