@@ -78,6 +78,16 @@ def aggregate_over_ranks(elapsed_ms: float, nbytes: int) -> Tuple[float, int]:
     return float(t.item()), int(b.item())
 
 
+L2_BYTES = 126 * 1000 * 1000
+
+
+def l2_note(state_bytes: int) -> str:
+    if state_bytes > 8 * L2_BYTES:
+        return f"inputs ({state_bytes / 1e9:.2f} GB) far larger than the 126 MB L2; no flush needed"
+    return (f"inputs ({state_bytes / 1e6:.1f} MB) fit the 126 MB L2 and no flush is done: these are L2- and "
+            "launch-bound numbers, not HBM numbers")
+
+
 def gbs(nbytes: float, ms: float) -> float:
     return nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
 
@@ -208,26 +218,37 @@ def oracle_sample_step(cfg, n_layers=1):
         keep = [i for i, s in enumerate(specs) if any(t in s.name for t in tags)]
         what = f"layers 0..{n_layers - 1} of every plane"
     host = [layouts.tensor_bytes(layouts._fill_model_tensor(cfg, specs[i], torch.device("cpu"))).numpy() for i in keep]
+    planes = [[j for j, i in enumerate(keep) if specs[i].plane == p] for p in (1, 2, 3)]
+    step, state_bytes = oracle_step_over(host, cfg.bucket_bytes, planes, 4, cfg.shard_r, cfg.shard_D)
+    sample = f"{what}: {len(keep)} tensors, {state_bytes / 1e9:.3f} GB of state, same four operations, shard r={cfg.shard_r} of {cfg.shard_D}"
+    return step, sample
+
+
+def oracle_step_over(host, bucket_bytes, planes, elem_size, r, D):
+    """A callable that runs the four oracle operations once over the host tensors `host` (shard of
+    every plane in `planes`, lists of indices into `host`) and returns (seconds, algorithmic bytes)."""
+    import numpy as np
+    import oracle
+    oracle.build()
     sizes = [h.size for h in host]
-    fp32 = {p: [j for j, i in enumerate(keep) if specs[i].plane == p] for p in (1, 2, 3)}
     state_bytes = sum(sizes)
-    _, total, nb = oracle.layout(sizes, cfg.bucket_bytes)
+    _, total, nb = oracle.layout(sizes, bucket_bytes)
     stream = np.empty(total, dtype=np.uint8)
 
     def step():
         t0 = time.perf_counter()
-        s, _ = oracle.pack(host, cfg.bucket_bytes, out=stream)
-        oracle.checksum(s, cfg.bucket_bytes)
+        s, _ = oracle.pack(host, bucket_bytes, out=stream)
+        oracle.checksum(s, bucket_bytes)
         oracle.unpack(s, sizes)
         shard_bytes = []
-        for p in (1, 2, 3):
-            out = oracle.shard([host[j] for j in fp32[p]], [sizes[j] for j in fp32[p]], 4, cfg.shard_r, cfg.shard_D)
-            shard_bytes.append(out.size)
+        for idx in planes:
+            if idx:
+                out = oracle.shard([host[j] for j in idx], [sizes[j] for j in idx], elem_size, r, D)
+                shard_bytes.append(out.size)
         dt = time.perf_counter() - t0
         return dt, sum(step_bytes(state_bytes, total, nb, shard_bytes).values())
 
-    sample = f"{what}: {len(keep)} tensors, {state_bytes / 1e9:.3f} GB of state, same four operations, shard r={cfg.shard_r} of {cfg.shard_D}"
-    return step, sample
+    return step, state_bytes
 
 
 def run_reference(args) -> None:
@@ -255,7 +276,9 @@ def run_reference(args) -> None:
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": len(times), "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8/u64", "data": "synthetic",
-        "config": {"workload": f"{args.workload}:{cfg.name}", "sample": sample},
+        "config": {"workload": f"{args.workload}:{cfg.name}", "sample": sample,
+                   "note": "the CPU oracle as it stands, one core, on a bounded one-layer sample of the workload "
+                           "(not the whole role); at most one warm-up step is run whatever --warmup says"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                          "host_cores_available": os.cpu_count()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -271,9 +294,9 @@ def run_reference(args) -> None:
 class RoleBench:
     """One role on the current GPU with every buffer the step needs."""
 
-    def __init__(self, workload: str, prepared=None):
+    def __init__(self, workload: str, prepared=None, layers: Optional[int] = None):
         from paper_2412_12636_b200 import layouts
-        from paper_2412_12636_b200.mover import MultiShardExtractor, RoleMover, ShardExtractor
+        from paper_2412_12636_b200.mover import MultiShardExtractor, RoleMover, ShardExtractor, ShardPlanMover
         if prepared is not None:      # (RoleState, bucket_bytes, r, D): a wave of a larger role
             self.state, self.bucket_bytes, self.shard_r, self.shard_D = prepared
             self.name = self.state.name
@@ -283,7 +306,7 @@ class RoleBench:
             self.name, self.bucket_bytes, self.shard_r, self.shard_D = "adversarial-20000", layouts.ADVERSARIAL_BUCKET, 29, 64
             planes = [self.state.elem_size_indices(4)]
         else:
-            cfg = layouts.role_config(WORKLOADS[workload])
+            cfg = layouts.role_config(WORKLOADS[workload], layers=layers)
             self.state = layouts.materialize(cfg, "cuda")
             self.name, self.bucket_bytes, self.shard_r, self.shard_D = cfg.name, cfg.bucket_bytes, cfg.shard_r, cfg.shard_D
             planes = [self.state.plane_indices(p) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)]
@@ -298,8 +321,12 @@ class RoleBench:
         for idx in planes:
             ex = ShardExtractor(self.target.descs_of(idx), self.shard_r, self.shard_D)
             self.shards.append((ex, ex.alloc_out()))
-        self.multi = MultiShardExtractor([self.target.descs_of(idx) for idx in planes], self.shard_r, self.shard_D)
         self.multi_outs = [out for _, out in self.shards]
+        plane_descs = [self.target.descs_of(idx) for idx in planes]
+        # the timed step runs the reusable plan (list built and uploaded once); the one-shot call, which
+        # rebuilds and uploads its list on every call, is timed beside it
+        self.shard_plan = ShardPlanMover(plane_descs, self.shard_r, self.shard_D, flats=self.multi_outs)
+        self.multi = MultiShardExtractor(plane_descs, self.shard_r, self.shard_D)
         self.per_op = step_bytes(state.state_bytes, self.mover.total_bytes, self.mover.n_buckets,
                                  [ex.out_bytes for ex, _ in self.shards])
         self.bytes_per_step = sum(self.per_op.values())
@@ -320,7 +347,7 @@ class RoleBench:
         mark()
         self.unmover.unpack(self.buckets)
         mark()
-        self.multi.extract(self.multi_outs)      # all planes' shards in one launch
+        self.shard_plan.extract()                # all planes' shards in one launch, no host work
         mark()
         if events is not None:
             events.append(marks)
@@ -353,6 +380,22 @@ class RoleBench:
         nbytes = self.per_op["unpack"] + 8 * self.mover.n_buckets
         return {"ms": round(ms, 4), "GB/s": round(gbs(nbytes, ms), 1),
                 "checksums_match": bool(torch.equal(got, self.cks_fused))}
+
+    def time_shard_one_shot(self, steps: int) -> Dict[str, float]:
+        """tm_shard_extract_planes (validates, builds and uploads its list on every call) against the
+        reusable plan of the timed step."""
+        outs = [torch.empty_like(o) for o in self.multi_outs]
+        for _ in range(2):
+            self.multi.extract(outs)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(self.stream)
+        for _ in range(steps):
+            self.multi.extract(outs)
+        b.record(self.stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / steps
+        same = all(torch.equal(o, m) for o, m in zip(outs, self.multi_outs))
+        return {"ms": round(ms, 4), "GB/s": round(gbs(self.per_op["shard"], ms), 1), "outputs_match": same}
 
     def time_pack_emit(self, steps: int):
         """tm_state_pack_emit (pack + the three fp32 shards in one launch) against pack, then shard."""
@@ -411,6 +454,7 @@ def run_config4_in_waves(args) -> None:
     sum_ms = {n: 0.0 for n in names}
     sum_bytes = {n: 0 for n in names}
     step_ms, step_bytes_total, ok, launches0 = 0.0, 0, True, binding.tm_launch_count()
+    cpu_baseline = None
     steps = max(2, min(args.steps, 5))
     for wi, w in enumerate(ws):
         wave_specs = [specs[p.tensor] for p in w.parts]
@@ -425,6 +469,23 @@ def run_config4_in_waves(args) -> None:
         torch.cuda.synchronize()
         ms, op_ms = role.timed(steps)
         ok = ok and role.self_check()
+        if wi == 0 and not args.no_cpu_baseline:
+            # the oracle, one core, on the first tensors of this wave (about 1.5 GB of state)
+            take, acc = [], 0
+            for k, t in enumerate(state.tensors):
+                if acc > 1_500_000_000:
+                    break
+                take.append(k)
+                acc += t.numel()
+            host = [state.host_bytes(k) for k in take]
+            fp32 = [j for j, k in enumerate(take) if state.specs[k].elem_size == 4]
+            ostep, sb = oracle_step_over(host, B, [fp32], 4, 29, layouts.ADVERSARIAL_D)
+            dt, nb_ = ostep()
+            cpu_baseline = {"value": round(gbs(nb_, dt * 1e3), 4), "unit": UNIT, "cores": 1, "kind": "oracle",
+                            "sample": f"first {len(take)} tensors of wave 0, {sb / 1e9:.3f} GB of state, same four operations, "
+                                      "shard r=29 of 64 over their fp32 tensors",
+                            "seconds": round(dt, 2), "host_cores_available": os.cpu_count()}
+            del host
         step_ms += ms / steps
         step_bytes_total += role.bytes_per_step
         for n in names:
@@ -442,7 +503,15 @@ def run_config4_in_waves(args) -> None:
                        "stream_bytes": total, "n_buckets": n_buckets, "bucket_bytes": B, "waves": len(ws),
                        "shard": "r=29 of D=64 over each wave's fp32 tensors",
                        "note": "processed in waves of whole buckets; ms_per_step is the sum over the waves"},
-            "bytes_per_step": step_bytes_total, "ops": ops, "roofline": None, "cpu_baseline": None, "e2e": None,
+            "bytes_per_step": step_bytes_total, "ops": ops,
+            "roofline": {"bound": "hbm", "kernel": "ring_kernel<pack> (fused pack + checksum), summed over the waves",
+                         "achieved": ops["pack"]["GB/s"], "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                         "frac": round(ops["pack"]["GB/s"] / peak, 4), "traffic": None,
+                         "traffic_note": "no counter capture of this layout", "algorithmic_bytes_per_launch": sum_bytes["pack"]},
+            "cpu_baseline": cpu_baseline,
+            "e2e": {"value": None, "unit": UNIT, "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+                    "skipped": "the 255 GB role does not fit pinned host memory next to its packed copy; "
+                               "the end-to-end leg is measured on cfg0..cfg3"},
             "gpu_launches": binding.tm_launch_count() - launches0, "self_check": "ok" if ok else "MISMATCH",
             "frac_of_measured_copy": round(gbs(step_bytes_total, step_ms) / peak, 4)}
     print(json.dumps(line), flush=True)
@@ -469,7 +538,7 @@ def run_ours(args) -> None:
     if use_dist:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    role = RoleBench(args.workload)
+    role = RoleBench(args.workload, layers=args.layers)
     for _ in range(max(args.warmup, 3)):
         role.one_step()
     torch.cuda.synchronize()
@@ -492,6 +561,8 @@ def run_ours(args) -> None:
     ok = ok and (fused_receive is None or fused_receive["checksums_match"])
     fused_send = role.time_pack_emit(max(3, args.steps // 2)) if rank == 0 else None
     ok = ok and (fused_send is None or fused_send["outputs_match"])
+    shard_one_shot = role.time_shard_one_shot(max(3, args.steps // 2)) if rank == 0 else None
+    ok = ok and (shard_one_shot is None or shard_one_shot["outputs_match"])
 
     total_ms, total_bytes = aggregate_over_ranks(elapsed_ms, role.bytes_per_step * args.steps)
     peak, peak_kind = measured_hbm_peak()
@@ -543,7 +614,7 @@ def run_ours(args) -> None:
         "config": {"workload": f"{args.workload}:{name}", "state_bytes": state_bytes,
                    "bucket_bytes": bucket_bytes, "n_buckets": n_buckets, "n_tensors": n_tensors,
                    "shard": f"{shard}, fp32 planes", "parallelism": "replicas only",
-                   "l2": "inputs (GBs) far larger than the 126 MB L2; no flush needed",
+                   "l2": l2_note(state_bytes),
                    "step": "pack+fused checksum, stand-alone checksum, unpack, shard extract of the three fp32 planes (one launch)"},
         "bytes_per_step": bytes_per_step, "ops": ops, "roofline": roofline, "cpu_baseline": cpu_baseline,
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "self_check": "ok" if ok else "MISMATCH",
@@ -552,8 +623,11 @@ def run_ours(args) -> None:
                                                 "buckets in one pass; not part of the timed step",
                                                 separate_ms=round(ops["checksum"]["ms"] + ops["unpack"]["ms"], 4)),
         "fused_send": fused_send and dict(fused_send, note="tm_state_pack_emit: pack + fused checksum + the three shards in one "
-                                          "launch; not part of the timed step",
+                                          "launch, every tensor read once; not part of the timed step",
+                                          pack_alone_ms=ops["pack"]["ms"],
                                           separate_ms=round(ops["pack"]["ms"] + ops["shard"]["ms"], 4)),
+        "shard_one_shot": shard_one_shot and dict(shard_one_shot, note="tm_shard_extract_planes: list built and uploaded on "
+                                                  "every call; the timed step uses the reusable tm_shard_plan"),
         "also": also,
     }
     print(json.dumps(line), flush=True)
@@ -601,8 +675,9 @@ def run_e2e(args, role):
         copied = 0   # tensors [0, copied) have their host->device copy enqueued
         up.wait_stream(compute)     # the previous step's readers of the tensors are done
         down.wait_stream(compute)
-        for i, w in enumerate(wm.waves):
+        for i in range(wm.n_waves):
             first, last = wm.tensor_ranges[i]
+            begin, end = wm.wave_span(i)
             with torch.cuda.stream(up):
                 for k in range(copied, last):
                     dev_bytes[k].copy_(views[k], non_blocking=True)
@@ -615,10 +690,10 @@ def run_e2e(args, role):
             packed.record(compute)
             with torch.cuda.stream(down):
                 down.wait_event(packed)
-                host_out[w.stream_begin:w.stream_end].copy_(buckets[w.stream_begin:w.stream_end], non_blocking=True)
+                host_out[begin:end].copy_(buckets[begin:end], non_blocking=True)
         role.mover.checksum(buckets, role.cks_alone)
         role.unmover.unpack(buckets)
-        role.multi.extract(role.multi_outs)
+        role.shard_plan.extract()
         o = mover.total_bytes
         host_out[o:o + 8 * mover.n_buckets].copy_(cks.view(torch.uint8), non_blocking=True)
         o += 8 * mover.n_buckets
@@ -646,8 +721,20 @@ def run_e2e(args, role):
     ms = s.elapsed_time(e) / k
     return {"value": round(gbs(role.bytes_per_step, max(ms, wall_ms)), 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": round(max(ms, wall_ms), 3), "steps": k,
-            "waves": len(wm.waves), "self_check": "ok" if ok else "MISMATCH",
+            "waves": wm.n_waves, "self_check": "ok" if ok else "MISMATCH",
             "note": "role tensors start and results end in pinned host memory; copies overlap the pack wave by wave; PCIe-bound"}
+
+
+def launch_local_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks on this node (one per GPU) through
+    torch.distributed.run with the same arguments; the ranks are independent replicas."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main() -> None:
@@ -660,7 +747,12 @@ def main() -> None:
     ap.add_argument("--also", default="cfg2", help="comma-separated further workloads measured after the main one (N=1 only); '' for none")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler launch lists)")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="reduce cfg0..cfg3 to their first LAYERS transformer layers: a small, self-ending case "
+                         "(a few GB, still far larger than the L2) for profiler captures")
     args = ap.parse_args()
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(launch_local_ranks(args.gpus))
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "cfg4":

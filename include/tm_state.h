@@ -49,11 +49,19 @@
  *     waiting; the caller synchronises.  The device of the stream/pointers must
  *     be the current device.
  *   - Every argument is validated on the host before anything is launched.
- *     Functions return TM_OK (0) or a negative tm_status.  On error nothing has
- *     been enqueued.  There is no CPU fallback: without a usable CUDA device
- *     the operations return TM_ERR_CUDA.
- *   - Calls are thread-safe with respect to one another, but one tm_plan must not
- *     be used by two threads at the same time.
+ *     Functions return TM_OK (0) or a negative tm_status.  On an argument error
+ *     nothing has been enqueued.  A TM_ERR_CUDA return means a runtime call failed
+ *     part-way: no kernel of the call has been launched, but a clearing memset or
+ *     a work-list upload may already sit in the stream.  There is no CPU fallback:
+ *     without a usable CUDA device the operations return TM_ERR_CUDA.
+ *   - Calls are thread-safe with respect to one another, but one plan object must
+ *     not be used by two threads at the same time.  tm_shard_extract_static has a
+ *     rule of its own (see there).
+ *   - An address named d_... only has to be readable / writable by the GPU: the
+ *     packed buffer (and, for that matter, the tensors) may live in mapped pinned
+ *     host memory, in which case the kernels move the bytes over PCIe themselves
+ *     (the "remote CPU memory checkpoint" tier of §7).  Checksum arrays and
+ *     workspaces should stay in device memory (the kernels update them with atomics).
  *   - Tensor addresses need only 2-byte alignment.  To serve such tensors at
  *     full speed the kernels read whole 16-byte-aligned lines: a line that
  *     holds at least one byte of a tensor may be read in full (it lies in the
@@ -79,7 +87,9 @@ typedef enum tm_status {
   TM_ERR_DTYPE    = -6,  /* elem_size not in {2,4,8}, or mixed elem_size inside one shard plane */
   TM_ERR_CUDA     = -7,  /* a CUDA runtime call failed (tm_last_cuda_error() gives its code) */
   TM_ERR_TIMEOUT  = -8,  /* a bounded device-side wait expired (reported by tm_plan_status / tm_workspace_status) */
-  TM_ERR_STATE    = -9   /* the plan has no uploaded work list (tm_plan_upload not called) */
+  TM_ERR_STATE    = -9,  /* the plan has no uploaded work list (tm_plan_upload / bind not called) */
+  TM_ERR_VERIFY   = -10, /* a transfer still had buckets with a checksum mismatch after the last round */
+  TM_ERR_TRANSPORT = -11 /* a transport or hook callback of a transfer returned non-zero */
 } tm_status;
 
 /* One tensor of a role's training state. */
@@ -92,21 +102,68 @@ typedef struct tm_desc {
 
 typedef struct tm_plan tm_plan;  /* opaque */
 
+/* ---- tuning ------------------------------------------------------------------------------- */
+
+/* Process-wide tuning values.  A plan keeps the values in force when it was created; launches read
+ * the rest from the plan.  The defaults are what every published number was measured with. */
+typedef struct tm_options {
+  uint64_t chunk_bytes;        /* largest piece of a pack / unpack plan; multiple of 256, 4 KiB .. 1 GiB; default 256 KiB */
+  uint64_t shard_chunk_bytes;  /* largest piece of a shard list (a shard is a fraction of a role); default 64 KiB */
+  uint64_t small_bytes;        /* pieces below this share a work item, one warp per piece; default 8 KiB */
+  uint64_t group_bytes;        /* byte budget of a shared item; default 64 KiB */
+  uint64_t cksum_tile_bytes;   /* tile of the stand-alone checksum kernel; multiple of 256; default 256 KiB */
+  uint64_t wait_limit_ns;      /* bound of every device-side wait of the ring kernels; 1 .. 5e9; default 2e9 */
+  uint32_t group_max;          /* piece budget of a shared item; 1 .. 1024; default 64 */
+  uint32_t ring_ctas_per_sm;   /* persistent blocks per SM of the ring kernels (96 KiB of shared memory each); 1 .. 2; default 1 */
+  uint32_t ctas_per_sm;        /* persistent blocks per SM of the checksum kernel; 1 .. 8; default 4 */
+  uint32_t reserved;           /* must be 0 */
+} tm_options;
+
+/* Reads the values in force. */
+int tm_options_get(tm_options* out);
+/* Replaces them (TM_ERR_ARG / TM_ERR_ALIGN if a value is out of range); NULL restores the defaults.
+ * Existing plans keep what they were built with. */
+int tm_options_set(const tm_options* in);
+
 /* ---- plan: layout of a role's tensors in the packed stream ------------------------------- */
 
 /* Computes the packed-stream layout (off_k, T, buckets; definitions above) for `n_desc`
  * descriptors and cuts it into the device work list.  Host only: no CUDA call is made.
  * `descs` is copied; it may be freed after the call.  *out receives a plan to be released with
  * tm_plan_destroy.  Errors: TM_ERR_ARG (NULL, n_desc == 0, nbytes == 0, nbytes % elem_size != 0,
- * bucket_bytes == 0 or > 2^35, nbytes > 2^46, n_desc > 2^24), TM_ERR_DTYPE, TM_ERR_ALIGN (odd ptr, bucket_bytes % 256 != 0). */
+ * bucket_bytes == 0 or > 2^35, nbytes > 2^46, n_desc > 2^24, T > 2^56), TM_ERR_DTYPE, TM_ERR_ALIGN
+ * (odd ptr, bucket_bytes % 256 != 0), TM_ERR_CAPACITY (out of host memory). */
 int tm_plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_plan** out);
+
+/* Plan for a run of whole buckets of the same stream — the unit in which a role travels through a
+ * bounded staging ring instead of a full second copy (§8.5 "Zero Memory Overhead Workflow": the
+ * channel is a recycled buffer, not a role-sized allocation).  The layout is computed for the
+ * complete descriptor list exactly as by tm_plan_create; the plan then covers stream bytes
+ * [first_bucket * B, min((first_bucket + n_buckets) * B, T)) only.  For such a plan the packed
+ * buffer passed to tm_state_pack / tm_state_unpack(_verify) / tm_state_pack_emit is a staging slot
+ * that holds just this range (its byte 0 is stream byte first_bucket * B; capacity >= the range's
+ * length, reported as total_bytes by tm_plan_query), and the checksum array has one entry per
+ * bucket of the range.  Buckets are independent units (each checksum restarts its word index), so the
+ * slots of consecutive ranges concatenate to the complete stream and their checksum arrays to the
+ * complete list.  Tensors outside the range are never touched (their ptr must still be non-NULL and
+ * even); a tensor that straddles a range boundary is split there.  first_bucket + n_buckets may
+ * exceed the bucket count (the range is clipped); first_bucket >= the bucket count is TM_ERR_ARG. */
+int tm_plan_create_range(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, uint64_t first_bucket,
+                         uint64_t n_buckets, tm_plan** out);
 
 /* Any of the three outputs may be NULL.  total_bytes = T, n_buckets = ceil(T/B),
  * workspace_bytes = size the caller must provide to tm_plan_upload. */
 int tm_plan_query(const tm_plan* plan, uint64_t* total_bytes, uint64_t* n_buckets,
                   uint64_t* workspace_bytes);
 
-/* Writes off_k for every descriptor into host array `offsets` (n_desc entries). */
+/* Where the plan sits in the complete stream (all outputs may be NULL): its first bucket, the stream
+ * offset of its first byte, and T and the bucket count of the complete stream.  For a plan made by
+ * tm_plan_create: 0, 0, and the same values as tm_plan_query. */
+int tm_plan_range(const tm_plan* plan, uint64_t* first_bucket, uint64_t* stream_begin, uint64_t* whole_bytes,
+                  uint64_t* whole_buckets);
+
+/* Writes off_k (offset in the complete stream) for every descriptor into host array `offsets`
+ * (n_desc entries). */
 int tm_plan_offsets(const tm_plan* plan, uint64_t* offsets);
 
 /* Copies the work list into caller-owned device memory `d_workspace` (256-byte aligned, at
@@ -150,16 +207,22 @@ int tm_state_unpack_verify(const tm_plan* plan, const void* d_buckets, uint64_t 
 
 /* Pack that also emits shards (the leaver, or a stayer holding a replica, hands a joiner both the
  * packed role and the slice of the optimizer state its data-parallel rank owns — §7 "State
- * Synchronization" — reading every tensor once).
+ * Synchronization" — and reads every tensor from memory once for both).
  *
  * tm_plan_attach_shards prepares it: planes are runs of the plan's own descriptors — plane p is
  * descriptors [plane_first_desc[p], + plane_n_desc[p]), runs ascending and disjoint, one elem_size
  * per plane — and each is sliced with the same r and D exactly as by tm_shard_extract, into
- * d_outs[p] (capacity out_capacities[p]).  The merged work list (every tensor's pack pieces followed
- * by the emit pieces that read the same tensor, so that the second read is served by the L2) is
- * uploaded once to d_workspace on `stream`.  With d_workspace == NULL nothing is uploaded and only
- * *workspace_needed (may be NULL otherwise) and out_elems (n_planes entries, may be NULL) are filled.
- * The outputs must not overlap the tensors, one another, or the packed buffer used later.
+ * d_outs[p] (capacity out_capacities[p]; the buffer receives the complete shard, element lo first).
+ * Every pack piece that holds shard elements gets a second destination for that sub-range; the
+ * kernel writes it from the same staged copy of the piece that feeds the stream and the checksum.
+ * (Pieces under 8 KiB are not staged; their few bytes are re-read through the caches.)  With a
+ * range plan only the part of each shard that lies in the plan's buckets is written, at its place in
+ * d_outs[p]; the plans of all ranges together fill the shard.  The list (pieces, items and emit
+ * records) is uploaded once to d_workspace on `stream`.  With d_workspace == NULL nothing is uploaded:
+ * *workspace_needed (may be NULL otherwise) and out_elems (n_planes entries, may be NULL) are filled,
+ * and if d_outs is given the emit records are computed for inspection (tm_plan_emits) while
+ * tm_state_pack_emit keeps returning TM_ERR_STATE.  The outputs must not overlap the tensors, one
+ * another, or the packed buffer used later.
  *
  * tm_state_pack_emit then does what tm_state_pack does (same arguments, same results) and fills the
  * attached shard outputs in the same launch. */
@@ -213,6 +276,35 @@ int tm_shard_insert(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uin
                     const void* d_in, uint64_t in_bytes, uint64_t* in_elems,
                     void* d_workspace, uint64_t workspace_bytes, void* stream);
 
+/* Reusable shard plan.  The one-shot calls above validate, build the work list on the host and
+ * upload it on every call; a plan does that once, after which extract and insert are single kernel
+ * launches with no host work (the joiner slices the same [lo, hi) out of master, m and v every time
+ * it is assigned a rank — §7 "State Synchronization").
+ *
+ * tm_shard_plan_create: `descs` is the concatenation of the planes' descriptor lists (plane p has
+ * plane_n_desc[p] entries, one elem_size per plane); validation and bounds as tm_shard_extract_planes.
+ * Host only.  tm_shard_plan_query: out_elems (n_planes entries, may be NULL) = hi - lo per plane;
+ * workspace_bytes (may be NULL) = device scratch tm_shard_plan_bind needs.
+ * tm_shard_plan_bind: fixes the flat buffers (d_flats[p], >= 2-byte aligned, capacities[p] >= the
+ * shard's bytes, no overlap with the tensors or one another; entries of empty shards are ignored),
+ * builds the list and uploads it to d_workspace (256-byte aligned) on `stream`.  May be called again
+ * to bind other buffers.  With d_workspace == NULL the list is only built (tm_shard_plan_pieces shows
+ * it) and extract / insert return TM_ERR_STATE.  tm_shard_plan_extract copies elements [lo, hi) of every plane to its flat
+ * buffer; tm_shard_plan_insert writes the flat buffers into elements [lo, hi) of the planes (the
+ * tensors of a plane must then not overlap one another: TM_ERR_OVERLAP).  Both are one launch, or none
+ * when every shard is empty. */
+typedef struct tm_shard_plan tm_shard_plan;
+int tm_shard_plan_create(const tm_desc* descs, const uint64_t* plane_n_desc, uint32_t n_planes, uint32_t r,
+                         uint32_t D, tm_shard_plan** out);
+int tm_shard_plan_query(const tm_shard_plan* sp, uint64_t* out_elems, uint64_t* workspace_bytes);
+int tm_shard_plan_bind(tm_shard_plan* sp, void* const* d_flats, const uint64_t* capacities, void* d_workspace,
+                       uint64_t workspace_bytes, void* stream);
+int tm_shard_plan_extract(const tm_shard_plan* sp, void* stream);
+int tm_shard_plan_insert(const tm_shard_plan* sp, void* stream);
+/* Status word of the plan's workspace (same meaning as tm_plan_status). */
+int tm_shard_plan_status(const tm_shard_plan* sp, void* stream, int* device_status);
+void tm_shard_plan_destroy(tm_shard_plan* sp);
+
 /* Size of the library-resident scratch array used by tm_shard_extract_static. */
 #define TM_STATIC_SCRATCH_BYTES (1u << 20)
 
@@ -229,8 +321,11 @@ int tm_shard_insert(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uin
  * device allocation and frees none.  The first call on each GPU resolves the array's device address
  * once, with that GPU current; make that call before starting any stream capture.  All calls on a
  * GPU share the array, which keeps the previous call's contents: the part that must start from zero
- * (the status block) is cleared on every call, and calls whose device work can overlap in time (two
- * streams, two threads) race on the list — serialise them on one stream. */
+ * (the status block) is cleared on every call.  The host side of a call (clear, two list copies,
+ * launch) runs under a lock, so calls from several threads on ONE stream are safe; calls whose
+ * device work can overlap in time (different streams) race on the list — issue them on one stream.
+ * The list is copied from ordinary host memory, so the call returns only after the stream has taken
+ * the copies (it may wait for earlier work in that stream). */
 int tm_shard_extract_static(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
                             void* d_out, uint64_t out_capacity, uint64_t* out_elems, void* stream);
 
@@ -269,6 +364,23 @@ typedef struct tm_piece {
  * (may be NULL) receive the full counts.  Host only. */
 int tm_plan_pieces(const tm_plan* plan, tm_piece* pieces, uint64_t capacity, uint64_t* n_pieces,
                    uint32_t* item_first, uint64_t item_capacity, uint64_t* n_items);
+
+/* Emit record of a piece after tm_plan_attach_shards: bytes [begin, begin + len) of the piece also go
+ * to device address `out`; len == 0 for pieces that hold no shard element. */
+typedef struct tm_emit {
+  uint64_t out;
+  uint32_t begin;
+  uint32_t len;
+} tm_emit;
+
+/* Copies the emit records (one per piece, in piece order) to `emits` (up to `capacity`); *n (may be
+ * NULL) receives the count — 0 before tm_plan_attach_shards.  Host only. */
+int tm_plan_emits(const tm_plan* plan, tm_emit* emits, uint64_t capacity, uint64_t* n);
+
+/* Work list of a bound shard plan, as tm_plan_pieces gives it for a plan; a piece's `off` is relative
+ * to *base (the lowest bound flat address; may be NULL), pad / bucket / word0 are 0.  Host only. */
+int tm_shard_plan_pieces(const tm_shard_plan* sp, tm_piece* pieces, uint64_t capacity, uint64_t* n_pieces,
+                         uint32_t* item_first, uint64_t item_capacity, uint64_t* n_items, uint64_t* base);
 
 /* ---- diagnostics ----------------------------------------------------------------------------- */
 

@@ -16,13 +16,27 @@ LIB_PATH = os.path.join(_HERE, "libtm_state.so")
 TM_OK = 0
 TM_ERR_ARG, TM_ERR_ALIGN, TM_ERR_CAPACITY, TM_ERR_OVERLAP = -1, -2, -3, -4
 TM_ERR_RANK, TM_ERR_DTYPE, TM_ERR_CUDA, TM_ERR_TIMEOUT, TM_ERR_STATE = -5, -6, -7, -8, -9
+TM_ERR_VERIFY, TM_ERR_TRANSPORT = -10, -11
 
 _u64, _u32, _p, _int = ctypes.c_uint64, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_int
 
 # every symbol include/tm_state.h declares: name -> (restype, argtypes)
 SIGNATURES = {
+    "tm_options_get": (_int, [_p]),
+    "tm_options_set": (_int, [_p]),
     "tm_plan_create": (_int, [_p, _u64, _u64, _p]),
+    "tm_plan_create_range": (_int, [_p, _u64, _u64, _u64, _u64, _p]),
     "tm_plan_query": (_int, [_p, _p, _p, _p]),
+    "tm_plan_range": (_int, [_p, _p, _p, _p, _p]),
+    "tm_plan_emits": (_int, [_p, _p, _u64, _p]),
+    "tm_shard_plan_create": (_int, [_p, _p, _u32, _u32, _u32, _p]),
+    "tm_shard_plan_query": (_int, [_p, _p, _p]),
+    "tm_shard_plan_bind": (_int, [_p, _p, _p, _p, _u64, _p]),
+    "tm_shard_plan_extract": (_int, [_p, _p]),
+    "tm_shard_plan_insert": (_int, [_p, _p]),
+    "tm_shard_plan_status": (_int, [_p, _p, _p]),
+    "tm_shard_plan_pieces": (_int, [_p, _p, _u64, _p, _p, _u64, _p, _p]),
+    "tm_shard_plan_destroy": (None, [_p]),
     "tm_plan_offsets": (_int, [_p, _p]),
     "tm_plan_pieces": (_int, [_p, _p, _u64, _p, _p, _u64, _p]),
     "tm_plan_upload": (_int, [_p, _p, _u64, _p]),
@@ -50,6 +64,12 @@ SIGNATURES = {
 
 class TmDesc(ctypes.Structure):
     _fields_ = [("ptr", _p), ("nbytes", _u64), ("elem_size", _u32), ("plane", _u32)]
+
+
+class TmOptions(ctypes.Structure):
+    _fields_ = [("chunk_bytes", _u64), ("shard_chunk_bytes", _u64), ("small_bytes", _u64), ("group_bytes", _u64),
+                ("cksum_tile_bytes", _u64), ("wait_limit_ns", _u64), ("group_max", _u32), ("ring_ctas_per_sm", _u32),
+                ("ctas_per_sm", _u32), ("reserved", _u32)]
 
 
 class TmError(RuntimeError):
@@ -94,19 +114,60 @@ def make_descs(descs: Iterable[Tuple[int, int, int, int]]):
     return arr
 
 
-class Plan:
-    """Owner of a tm_plan handle."""
+def tm_options_get() -> dict:
+    o = TmOptions()
+    _check(load_library().tm_options_get(ctypes.byref(o)), "tm_options_get")
+    return {name: getattr(o, name) for name, _ in TmOptions._fields_ if name != "reserved"}
 
-    def __init__(self, descs: Sequence[Tuple[int, int, int, int]], bucket_bytes: int):
+
+def tm_options_set(**values) -> None:
+    """Sets the named tuning values (the others keep their current value); no arguments restores the
+    defaults.  Plans created afterwards use them."""
+    L = load_library()
+    if not values:
+        _check(L.tm_options_set(None), "tm_options_set")
+        return
+    o = TmOptions()
+    _check(L.tm_options_get(ctypes.byref(o)), "tm_options_get")
+    for k, v in values.items():
+        setattr(o, k, v)
+    _check(L.tm_options_set(ctypes.byref(o)), "tm_options_set")
+
+
+_PIECE_DTYPE = [("tensor", "<u8"), ("off", "<u8"), ("nbytes", "<u4"), ("pad", "<u4"), ("bucket", "<u4"), ("word0", "<u4")]
+
+
+class Plan:
+    """Owner of a tm_plan handle.  With `first_bucket` / `n_buckets` the plan covers that run of whole
+    buckets of the stream only (tm_plan_create_range)."""
+
+    def __init__(self, descs, bucket_bytes: int, first_bucket: Optional[int] = None, n_buckets: Optional[int] = None):
         L = load_library()
         self._h = _p()
-        arr = make_descs(descs)
-        _check(L.tm_plan_create(arr, len(arr), bucket_bytes, ctypes.byref(self._h)), "tm_plan_create")
+        arr = descs if isinstance(descs, ctypes.Array) else make_descs(descs)
+        if first_bucket is None:
+            _check(L.tm_plan_create(arr, len(arr), bucket_bytes, ctypes.byref(self._h)), "tm_plan_create")
+        else:
+            _check(L.tm_plan_create_range(arr, len(arr), bucket_bytes, first_bucket, n_buckets, ctypes.byref(self._h)),
+                   "tm_plan_create_range")
         self.n_desc = len(arr)
         t, n, w = _u64(), _u64(), _u64()
         _check(L.tm_plan_query(self._h, ctypes.byref(t), ctypes.byref(n), ctypes.byref(w)), "tm_plan_query")
         self.total_bytes, self.n_buckets, self.workspace_bytes = t.value, n.value, w.value
+        f, b, wt, wn = _u64(), _u64(), _u64(), _u64()
+        _check(L.tm_plan_range(self._h, ctypes.byref(f), ctypes.byref(b), ctypes.byref(wt), ctypes.byref(wn)), "tm_plan_range")
+        self.first_bucket, self.stream_begin, self.whole_bytes, self.whole_buckets = f.value, b.value, wt.value, wn.value
         self.bucket_bytes = bucket_bytes
+
+    def emits(self):
+        """Emit records (numpy array with fields out, begin, len), one per piece; empty before attach."""
+        import numpy as np
+        L = load_library()
+        n = _u64()
+        _check(L.tm_plan_emits(self._h, None, 0, ctypes.byref(n)), "tm_plan_emits")
+        out = np.zeros(n.value, dtype=np.dtype([("out", "<u8"), ("begin", "<u4"), ("len", "<u4")]))
+        _check(L.tm_plan_emits(self._h, out.ctypes.data, out.size, None), "tm_plan_emits")
+        return out
 
     def offsets(self) -> List[int]:
         out = (_u64 * self.n_desc)()
@@ -120,9 +181,7 @@ class Plan:
         L = load_library()
         np_, ni = _u64(), _u64()
         _check(L.tm_plan_pieces(self._h, None, 0, ctypes.byref(np_), None, 0, ctypes.byref(ni)), "tm_plan_pieces")
-        dt = np.dtype([("tensor", "<u8"), ("off", "<u8"), ("nbytes", "<u4"), ("pad", "<u4"), ("bucket", "<u4"),
-                       ("word0", "<u4")])
-        pieces = np.zeros(np_.value, dtype=dt)
+        pieces = np.zeros(np_.value, dtype=np.dtype(_PIECE_DTYPE))
         items = np.zeros(ni.value + 1, dtype=np.uint32)
         _check(L.tm_plan_pieces(self._h, pieces.ctypes.data, pieces.size, None, items.ctypes.data, items.size, None),
                "tm_plan_pieces")
@@ -231,6 +290,65 @@ def tm_shard_insert(descs, r: int, D: int, d_in: int, in_bytes: int, d_workspace
     _check(load_library().tm_shard_insert(arr, len(arr), r, D, d_in, in_bytes, ctypes.byref(n), d_workspace,
                                           workspace_bytes, stream), "tm_shard_insert")
     return n.value
+
+
+class ShardPlan:
+    """Owner of a tm_shard_plan handle: shard r of D of one or several planes, bound once to its flat
+    buffers, then extract / insert are single launches."""
+
+    def __init__(self, planes, r: int, D: int):
+        L = load_library()
+        self._h = _p()
+        self.n_planes = len(planes)
+        arr = make_descs([d for plane in planes for d in plane])
+        counts = (_u64 * self.n_planes)(*[len(p) for p in planes])
+        _check(L.tm_shard_plan_create(arr, counts, self.n_planes, r, D, ctypes.byref(self._h)), "tm_shard_plan_create")
+        got, w = (_u64 * self.n_planes)(), _u64()
+        _check(L.tm_shard_plan_query(self._h, got, ctypes.byref(w)), "tm_shard_plan_query")
+        self.elems, self.workspace_bytes = list(got), w.value
+        self.out_bytes = [n * plane[0][2] for n, plane in zip(self.elems, planes)]
+
+    def bind(self, d_flats: Sequence[int], capacities: Sequence[int], d_workspace: int, workspace_bytes: int,
+             stream: int) -> None:
+        flats = (_p * self.n_planes)(*d_flats)
+        caps = (_u64 * self.n_planes)(*capacities)
+        _check(load_library().tm_shard_plan_bind(self._h, flats, caps, d_workspace, workspace_bytes, stream),
+               "tm_shard_plan_bind")
+
+    def extract(self, stream: int) -> None:
+        _check(load_library().tm_shard_plan_extract(self._h, stream), "tm_shard_plan_extract")
+
+    def insert(self, stream: int) -> None:
+        _check(load_library().tm_shard_plan_insert(self._h, stream), "tm_shard_plan_insert")
+
+    def status(self, stream: int) -> int:
+        s = _int()
+        _check(load_library().tm_shard_plan_status(self._h, stream, ctypes.byref(s)), "tm_shard_plan_status")
+        return s.value
+
+    def pieces(self):
+        """(pieces, item_first, base): the bound work list; piece offsets are relative to `base`."""
+        import numpy as np
+        L = load_library()
+        np_, ni, base = _u64(), _u64(), _u64()
+        _check(L.tm_shard_plan_pieces(self._h, None, 0, ctypes.byref(np_), None, 0, ctypes.byref(ni), ctypes.byref(base)),
+               "tm_shard_plan_pieces")
+        pieces = np.zeros(np_.value, dtype=np.dtype(_PIECE_DTYPE))
+        items = np.zeros(ni.value + 1, dtype=np.uint32)
+        _check(L.tm_shard_plan_pieces(self._h, pieces.ctypes.data, pieces.size, None, items.ctypes.data, items.size,
+                                      None, None), "tm_shard_plan_pieces")
+        return pieces, items, base.value
+
+    def close(self) -> None:
+        if self._h:
+            load_library().tm_shard_plan_destroy(self._h)
+            self._h = _p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def tm_shard_extract_static(descs, r: int, D: int, d_out: int, out_capacity: int, stream: int) -> int:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtm_state.so")
-SOURCES = [os.path.join(CSRC, f) for f in ("kernels.cu", "plan.cpp", "api.cpp", "static_scratch.cu", "ring_kernels.cu")]
+SOURCES = [os.path.join(CSRC, f) for f in ("kernels.cu", "plan.cpp", "api.cpp", "shard.cpp", "transfer.cpp", "static_scratch.cu", "ring_kernels.cu")]
 HEADERS = [os.path.join(CSRC, "tm_internal.h"), os.path.join(CSRC, "device_util.cuh"), os.path.join(ROOT, "include", "tm_state.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]

@@ -12,32 +12,36 @@
 
 #include "tm_internal.h"
 
-int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes);
-int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
-int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_t D,
-                      uint32_t* elem_size, uint64_t* n_elems);
-void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
-                       uint64_t d_out, tms::WorkList* wl);
-int tm_targets_disjoint(const tm_plan* p);
-void tm_shard_append(tms::WorkListBuilder* builder, const tm_desc* descs, uint64_t n_desc, uint32_t e,
-                     uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base, uint32_t bucket_tag);
-
 namespace {
 
 std::atomic<int> g_last_cuda_error{0};
 
-int cuda_fail(int e) {
-  g_last_cuda_error.store(e);
-  return TM_ERR_CUDA;
-}
-#define TM_CUDA(call)                              \
-  do {                                             \
-    cudaError_t e__ = (call);                      \
-    if (e__ != cudaSuccess) return cuda_fail((int)e__); \
+#define TM_CUDA(call)                                   \
+  do {                                                  \
+    cudaError_t e__ = (call);                           \
+    if (e__ != cudaSuccess) return tms::cuda_fail((int)e__); \
   } while (0)
 
-bool ranges_overlap(uint64_t a, uint64_t an, uint64_t b, uint64_t bn) {
-  return a < b + bn && b < a + an;
+// No C++ exception may cross the C boundary: host allocations that fail become TM_ERR_CAPACITY.
+template <typename F>
+int guarded(F&& f) noexcept {
+  try {
+    return f();
+  } catch (const std::bad_alloc&) {
+    return TM_ERR_CAPACITY;
+  } catch (...) {
+    return TM_ERR_ARG;
+  }
+}
+
+// True when the packed buffer [base, base + nbytes) overlaps a tensor part the plan touches.  The
+// plan's address bounding box settles the common case without walking the parts.
+bool plan_overlaps(const tm_plan* plan, uint64_t base, uint64_t nbytes) {
+  if (plan->box_hi <= plan->box_lo || !tms::ranges_overlap(plan->box_lo, plan->box_hi - plan->box_lo, base, nbytes))
+    return false;
+  for (const tm_part& q : plan->parts)
+    if (tms::ranges_overlap(q.addr, q.nbytes, base, nbytes)) return true;
+  return false;
 }
 
 // Pinned host staging for small work-list uploads: eight 1 MiB slots per device, reused round-robin;
@@ -93,10 +97,23 @@ class HostStaging {
 };
 HostStaging g_staging;
 
-int upload_worklist(const tms::WorkList& wl, const tms::WorkspaceLayout& l, uint8_t* d_ws, cudaStream_t st) {
+}  // namespace
+
+namespace tms {
+
+int cuda_fail(int e) {
+  g_last_cuda_error.store(e);
+  return TM_ERR_CUDA;
+}
+
+int upload_worklist(const WorkList& wl, const std::vector<Emit>* emits, const WorkspaceLayout& l, uint8_t* d_ws,
+                    void* stream) {
+  cudaStream_t st = (cudaStream_t)stream;
   const size_t items_bytes = wl.item_first.size() * sizeof(uint32_t);
-  const size_t segs_bytes = wl.segs.size() * sizeof(tms::Seg);
-  const size_t span = l.items_off + items_bytes;   // status block, pieces, items: one contiguous image
+  const size_t segs_bytes = wl.segs.size() * sizeof(Seg);
+  const size_t emits_bytes = emits != nullptr ? emits->size() * sizeof(Emit) : 0;
+  // status block, pieces, items (, emit records): one contiguous image
+  const size_t span = emits != nullptr ? l.emits_off + emits_bytes : l.items_off + items_bytes;
   if (span <= HostStaging::kSlotBytes) {
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) {
@@ -104,25 +121,28 @@ int upload_worklist(const tms::WorkList& wl, const tms::WorkspaceLayout& l, uint
       const int slot = g_staging.acquire(dev);
       if (slot >= 0) {
         uint8_t* h = g_staging.host(dev, slot);
-        std::memset(h, 0, l.segs_off);
+        std::memset(h, 0, span);
         if (segs_bytes != 0) std::memcpy(h + l.segs_off, wl.segs.data(), segs_bytes);
-        std::memset(h + l.segs_off + segs_bytes, 0, l.items_off - l.segs_off - segs_bytes);
         std::memcpy(h + l.items_off, wl.item_first.data(), items_bytes);
+        if (emits_bytes != 0) std::memcpy(h + l.emits_off, emits->data(), emits_bytes);
         TM_CUDA(cudaMemcpyAsync(d_ws, h, span, cudaMemcpyHostToDevice, st));
         TM_CUDA(g_staging.mark(dev, slot, st));
         return TM_OK;
       }
     }
   }
-  TM_CUDA(cudaMemsetAsync(d_ws, 0, tms::kStatusBlockBytes, st));
+  TM_CUDA(cudaMemsetAsync(d_ws, 0, kStatusBlockBytes, st));
   if (segs_bytes != 0)
     TM_CUDA(cudaMemcpyAsync(d_ws + l.segs_off, wl.segs.data(), segs_bytes, cudaMemcpyHostToDevice, st));
   TM_CUDA(cudaMemcpyAsync(d_ws + l.items_off, wl.item_first.data(), items_bytes, cudaMemcpyHostToDevice, st));
+  if (emits_bytes != 0)
+    TM_CUDA(cudaMemcpyAsync(d_ws + l.emits_off, emits->data(), emits_bytes, cudaMemcpyHostToDevice, st));
   return TM_OK;
 }
 
-int read_status(const void* d_ws, cudaStream_t st, int* device_status) {
+int read_status_word(const void* d_ws, void* stream, int* device_status) {
   if (d_ws == nullptr || device_status == nullptr) return TM_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
   int word = 0;
   TM_CUDA(cudaMemcpyAsync(&word, d_ws, sizeof(int), cudaMemcpyDeviceToHost, st));
   TM_CUDA(cudaStreamSynchronize(st));
@@ -130,22 +150,74 @@ int read_status(const void* d_ws, cudaStream_t st, int* device_status) {
   return TM_OK;
 }
 
+}  // namespace tms
+
+namespace {
+
+tms::RingLaunch ring_args(const tm_plan* plan, const uint8_t* ws, const tms::WorkspaceLayout& l, void* d_buckets,
+                          uint64_t* d_checksums) {
+  tms::RingLaunch a;
+  a.d_segs = (const tms::Seg*)(ws + l.segs_off);
+  a.d_item_first = (const uint32_t*)(ws + l.items_off);
+  a.n_items = (uint32_t)plan->work.n_items();
+  a.d_flat = (uint8_t*)d_buckets;
+  a.d_checksums = (unsigned long long*)d_checksums;
+  a.d_status = (int*)const_cast<uint8_t*>(ws);
+  a.wait_limit_ns = plan->opt.wait_limit_ns;
+  a.ctas_per_sm = plan->opt.ring_ctas_per_sm;
+  return a;
+}
+
+// Checks shared by pack, pack_emit, unpack and unpack_verify.
+int check_buckets(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, const void* d_checksums) {
+  if (plan == nullptr || d_buckets == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_buckets & 255) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
+  if (nbytes < plan->total_bytes) return TM_ERR_CAPACITY;
+  if (plan_overlaps(plan, (uint64_t)(uintptr_t)d_buckets, plan->total_bytes)) return TM_ERR_OVERLAP;
+  return TM_OK;
+}
+
 }  // namespace
 
 extern "C" {
 
-int tm_plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_plan** out) {
+int tm_options_get(tm_options* out) {
+  if (out == nullptr) return TM_ERR_ARG;
+  *out = tms::tuning();
+  return TM_OK;
+}
+
+int tm_options_set(const tm_options* in) { return tms::set_tuning(in); }
+
+static int plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, bool ranged, uint64_t first,
+                       uint64_t count, tm_plan** out) {
   if (out == nullptr) return TM_ERR_ARG;
   *out = nullptr;
-  tm_plan* p = new (std::nothrow) tm_plan();
-  if (p == nullptr) return TM_ERR_ARG;
-  int rc = tm_plan_build(p, descs, n_desc, bucket_bytes);
-  if (rc != TM_OK) {
-    delete p;
-    return rc;
-  }
-  *out = p;
-  return TM_OK;
+  return guarded([&]() -> int {
+    tm_plan* p = new tm_plan();
+    int rc = TM_ERR_CAPACITY;
+    try {
+      rc = tm_plan_build(p, descs, n_desc, bucket_bytes, ranged, first, count);
+    } catch (...) {
+      delete p;
+      throw;
+    }
+    if (rc != TM_OK) {
+      delete p;
+      return rc;
+    }
+    *out = p;
+    return TM_OK;
+  });
+}
+
+int tm_plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_plan** out) {
+  return plan_create(descs, n_desc, bucket_bytes, false, 0, 0, out);
+}
+
+int tm_plan_create_range(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, uint64_t first_bucket,
+                         uint64_t n_buckets, tm_plan** out) {
+  return plan_create(descs, n_desc, bucket_bytes, true, first_bucket, n_buckets, out);
 }
 
 int tm_plan_query(const tm_plan* plan, uint64_t* total_bytes, uint64_t* n_buckets,
@@ -157,22 +229,53 @@ int tm_plan_query(const tm_plan* plan, uint64_t* total_bytes, uint64_t* n_bucket
   return TM_OK;
 }
 
+int tm_plan_range(const tm_plan* plan, uint64_t* first_bucket, uint64_t* stream_begin, uint64_t* whole_bytes,
+                  uint64_t* whole_buckets) {
+  if (plan == nullptr) return TM_ERR_ARG;
+  if (first_bucket != nullptr) *first_bucket = plan->first_bucket;
+  if (stream_begin != nullptr) *stream_begin = plan->range_begin;
+  if (whole_bytes != nullptr) *whole_bytes = plan->whole_bytes;
+  if (whole_buckets != nullptr) *whole_buckets = plan->whole_buckets;
+  return TM_OK;
+}
+
 int tm_plan_offsets(const tm_plan* plan, uint64_t* offsets) {
   if (plan == nullptr || offsets == nullptr) return TM_ERR_ARG;
   std::memcpy(offsets, plan->offsets.data(), plan->offsets.size() * sizeof(uint64_t));
   return TM_OK;
 }
 
+static int copy_pieces(const tms::WorkList& wl, tm_piece* pieces, uint64_t capacity, uint64_t* n_pieces,
+                       uint32_t* item_first, uint64_t item_capacity, uint64_t* n_items) {
+  static_assert(sizeof(tm_piece) == sizeof(tms::Seg), "tm_piece mirrors the internal piece");
+  const uint64_t np = wl.segs.size(), ni = wl.n_items();
+  if (n_pieces != nullptr) *n_pieces = np;
+  if (n_items != nullptr) *n_items = ni;
+  if (pieces != nullptr) std::memcpy(pieces, wl.segs.data(), std::min(np, capacity) * sizeof(tm_piece));
+  if (item_first != nullptr && !wl.item_first.empty())
+    std::memcpy(item_first, wl.item_first.data(), std::min(ni + 1, item_capacity) * sizeof(uint32_t));
+  return TM_OK;
+}
+
 int tm_plan_pieces(const tm_plan* plan, tm_piece* pieces, uint64_t capacity, uint64_t* n_pieces,
                    uint32_t* item_first, uint64_t item_capacity, uint64_t* n_items) {
   if (plan == nullptr) return TM_ERR_ARG;
-  static_assert(sizeof(tm_piece) == sizeof(tms::Seg), "tm_piece mirrors the internal piece");
-  const uint64_t np = plan->work.segs.size(), ni = plan->work.n_items();
-  if (n_pieces != nullptr) *n_pieces = np;
-  if (n_items != nullptr) *n_items = ni;
-  if (pieces != nullptr) std::memcpy(pieces, plan->work.segs.data(), std::min(np, capacity) * sizeof(tm_piece));
-  if (item_first != nullptr)
-    std::memcpy(item_first, plan->work.item_first.data(), std::min(ni + 1, item_capacity) * sizeof(uint32_t));
+  return copy_pieces(plan->work, pieces, capacity, n_pieces, item_first, item_capacity, n_items);
+}
+
+int tm_shard_plan_pieces(const tm_shard_plan* sp, tm_piece* pieces, uint64_t capacity, uint64_t* n_pieces,
+                         uint32_t* item_first, uint64_t item_capacity, uint64_t* n_items, uint64_t* base) {
+  if (sp == nullptr) return TM_ERR_ARG;
+  if (base != nullptr) *base = sp->base;
+  return copy_pieces(sp->work, pieces, capacity, n_pieces, item_first, item_capacity, n_items);
+}
+
+int tm_plan_emits(const tm_plan* plan, tm_emit* emits, uint64_t capacity, uint64_t* n) {
+  if (plan == nullptr) return TM_ERR_ARG;
+  static_assert(sizeof(tm_emit) == sizeof(tms::Emit), "tm_emit mirrors the internal record");
+  if (n != nullptr) *n = plan->emits.size();
+  if (emits != nullptr)
+    std::memcpy(emits, plan->emits.data(), std::min<uint64_t>(plan->emits.size(), capacity) * sizeof(tm_emit));
   return TM_OK;
 }
 
@@ -180,7 +283,7 @@ int tm_plan_upload(tm_plan* plan, void* d_workspace, uint64_t workspace_bytes, v
   if (plan == nullptr || d_workspace == nullptr) return TM_ERR_ARG;
   if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
   if (workspace_bytes < plan->ws_layout.total) return TM_ERR_CAPACITY;
-  int rc = upload_worklist(plan->work, plan->ws_layout, (uint8_t*)d_workspace, (cudaStream_t)stream);
+  int rc = tms::upload_worklist(plan->work, nullptr, plan->ws_layout, (uint8_t*)d_workspace, stream);
   if (rc != TM_OK) return rc;
   plan->d_workspace = (uint8_t*)d_workspace;
   return TM_OK;
@@ -191,11 +294,11 @@ int tm_plan_status(const tm_plan* plan, void* stream, int* device_status) {
   if (plan->d_workspace == nullptr && plan->d_emit_workspace == nullptr) return TM_ERR_STATE;
   int a = 0, b = 0;
   if (plan->d_workspace != nullptr) {
-    int rc = read_status(plan->d_workspace, (cudaStream_t)stream, &a);
+    int rc = tms::read_status_word(plan->d_workspace, stream, &a);
     if (rc != TM_OK) return rc;
   }
   if (plan->d_emit_workspace != nullptr) {
-    int rc = read_status(plan->d_emit_workspace, (cudaStream_t)stream, &b);
+    int rc = tms::read_status_word(plan->d_emit_workspace, stream, &b);
     if (rc != TM_OK) return rc;
   }
   *device_status = (a != 0) ? a : b;
@@ -206,94 +309,82 @@ void tm_plan_destroy(tm_plan* plan) { delete plan; }
 
 int tm_state_pack(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint64_t* d_checksums,
                   void* stream) {
-  if (plan == nullptr || d_buckets == nullptr) return TM_ERR_ARG;
+  int rc = check_buckets(plan, d_buckets, capacity, d_checksums);
+  if (rc != TM_OK) return rc;
   if (plan->d_workspace == nullptr) return TM_ERR_STATE;
-  if (((uintptr_t)d_buckets & 255) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
-  if (capacity < plan->total_bytes) return TM_ERR_CAPACITY;
-  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
-  for (const tm_desc& d : plan->descs)
-    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
-  cudaStream_t st = (cudaStream_t)stream;
   if (d_checksums != nullptr)
-    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), st));
-  const uint8_t* ws = plan->d_workspace;
-  auto pack_fn = tms::tuning().use_ring ? tms::launch_pack_ring : tms::launch_pack;
-  int e = pack_fn((const tms::Seg*)(ws + plan->ws_layout.segs_off),
-                          (const uint32_t*)(ws + plan->ws_layout.items_off),
-                          (uint32_t)plan->work.n_items(), (uint8_t*)d_buckets,
-                          (unsigned long long*)d_checksums, (int*)plan->d_workspace, stream);
-  return e == 0 ? TM_OK : cuda_fail(e);
+    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), (cudaStream_t)stream));
+  int e = tms::launch_ring(tms::kRingPack, ring_args(plan, plan->d_workspace, plan->ws_layout, d_buckets, d_checksums),
+                           stream);
+  return e == 0 ? TM_OK : tms::cuda_fail(e);
+}
+
+static int targets_ok(const tm_plan* plan) {
+  if (plan->targets_disjoint == 0) plan->targets_disjoint = tm_parts_disjoint(plan->parts);
+  return plan->targets_disjoint < 0 ? TM_ERR_OVERLAP : TM_OK;
 }
 
 int tm_state_unpack(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, void* stream) {
-  if (plan == nullptr || d_buckets == nullptr) return TM_ERR_ARG;
-  if (plan->d_workspace == nullptr) return TM_ERR_STATE;
-  if (((uintptr_t)d_buckets & 255) != 0) return TM_ERR_ALIGN;
-  if (nbytes < plan->total_bytes) return TM_ERR_CAPACITY;
-  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
-  for (const tm_desc& d : plan->descs)
-    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
-  if (plan->targets_disjoint == 0) plan->targets_disjoint = tm_targets_disjoint(plan);
-  if (plan->targets_disjoint < 0) return TM_ERR_OVERLAP;
-  const uint8_t* ws = plan->d_workspace;
-  auto copy_fn = tms::tuning().use_ring ? tms::launch_copy_ring : tms::launch_copy;
-  int e = copy_fn((const tms::Seg*)(ws + plan->ws_layout.segs_off),
-                          (const uint32_t*)(ws + plan->ws_layout.items_off),
-                          (uint32_t)plan->work.n_items(), (uint8_t*)const_cast<void*>(d_buckets),
-                          /*to_tensors=*/true, (int*)plan->d_workspace, stream);
-  return e == 0 ? TM_OK : cuda_fail(e);
+  return guarded([&]() -> int {
+    int rc = check_buckets(plan, d_buckets, nbytes, nullptr);
+    if (rc != TM_OK) return rc;
+    if (plan->d_workspace == nullptr) return TM_ERR_STATE;
+    if ((rc = targets_ok(plan)) != TM_OK) return rc;
+    int e = tms::launch_ring(tms::kRingToTensors,
+                             ring_args(plan, plan->d_workspace, plan->ws_layout, const_cast<void*>(d_buckets), nullptr),
+                             stream);
+    return e == 0 ? TM_OK : tms::cuda_fail(e);
+  });
 }
 
 int tm_state_unpack_verify(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, uint64_t* d_checksums,
                            void* stream) {
-  if (plan == nullptr || d_buckets == nullptr || d_checksums == nullptr) return TM_ERR_ARG;
-  if (plan->d_workspace == nullptr) return TM_ERR_STATE;
-  if (((uintptr_t)d_buckets & 255) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
-  if (nbytes < plan->total_bytes) return TM_ERR_CAPACITY;
-  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
-  for (const tm_desc& d : plan->descs)
-    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
-  if (plan->targets_disjoint == 0) plan->targets_disjoint = tm_targets_disjoint(plan);
-  if (plan->targets_disjoint < 0) return TM_ERR_OVERLAP;
-  TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), (cudaStream_t)stream));
-  const uint8_t* ws = plan->d_workspace;
-  int e = tms::launch_unpack_verify_ring((const tms::Seg*)(ws + plan->ws_layout.segs_off),
-                                         (const uint32_t*)(ws + plan->ws_layout.items_off),
-                                         (uint32_t)plan->work.n_items(), (uint8_t*)const_cast<void*>(d_buckets),
-                                         (unsigned long long*)d_checksums, (int*)plan->d_workspace, stream);
-  return e == 0 ? TM_OK : cuda_fail(e);
+  return guarded([&]() -> int {
+    if (d_checksums == nullptr) return TM_ERR_ARG;
+    int rc = check_buckets(plan, d_buckets, nbytes, d_checksums);
+    if (rc != TM_OK) return rc;
+    if (plan->d_workspace == nullptr) return TM_ERR_STATE;
+    if ((rc = targets_ok(plan)) != TM_OK) return rc;
+    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), (cudaStream_t)stream));
+    int e = tms::launch_ring(tms::kRingToTensorsVerify,
+                             ring_args(plan, plan->d_workspace, plan->ws_layout, const_cast<void*>(d_buckets), d_checksums),
+                             stream);
+    return e == 0 ? TM_OK : tms::cuda_fail(e);
+  });
 }
 
 int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const uint64_t* plane_n_desc,
                           uint32_t n_planes, uint32_t r, uint32_t D, void* const* d_outs,
                           const uint64_t* out_capacities, uint64_t* out_elems, void* d_workspace,
                           uint64_t workspace_bytes, uint64_t* workspace_needed, void* stream) {
-  if (plan == nullptr || plane_first_desc == nullptr || plane_n_desc == nullptr || n_planes == 0)
-    return TM_ERR_ARG;
-  if (D == 0 || r >= D) return TM_ERR_RANK;
-  const uint64_t n_desc = plan->descs.size();
-  struct PlaneInfo { uint64_t first, n; uint32_t e; uint64_t lo, hi; };
-  std::vector<PlaneInfo> planes(n_planes);
-  uint64_t prev_end = 0;
-  for (uint32_t p = 0; p < n_planes; ++p) {
-    PlaneInfo& pi = planes[p];
-    pi.first = plane_first_desc[p];
-    pi.n = plane_n_desc[p];
-    if (pi.n == 0 || pi.first < prev_end || pi.first + pi.n > n_desc) return TM_ERR_ARG;   // ascending, disjoint
-    prev_end = pi.first + pi.n;
-    uint64_t n_elems = 0;
-    int rc = tm_shard_validate(plan->descs.data() + pi.first, pi.n, r, D, &pi.e, &n_elems);
-    if (rc != TM_OK) return rc;
-    rc = tm_bounds_u128(n_elems, r, D, &pi.lo, &pi.hi);
-    if (rc != TM_OK) return rc;
-    if (out_elems != nullptr) out_elems[p] = pi.hi - pi.lo;
-  }
-  const bool dry = (d_workspace == nullptr);
-  uint64_t base = ~0ull;
-  std::vector<std::pair<uint64_t, uint64_t>> outs;
-  if (!dry) {
+  return guarded([&]() -> int {
+    if (plan == nullptr || plane_first_desc == nullptr || plane_n_desc == nullptr || n_planes == 0)
+      return TM_ERR_ARG;
+    if (D == 0 || r >= D) return TM_ERR_RANK;
+    const uint64_t n_desc = plan->descs.size();
+    struct PlaneInfo { uint64_t first, n; uint32_t e; uint64_t lo, hi; };
+    std::vector<PlaneInfo> planes(n_planes);
+    uint64_t prev_end = 0;
+    for (uint32_t p = 0; p < n_planes; ++p) {
+      PlaneInfo& pi = planes[p];
+      pi.first = plane_first_desc[p];
+      pi.n = plane_n_desc[p];
+      if (pi.n == 0 || pi.first < prev_end || pi.n > n_desc || pi.first > n_desc - pi.n) return TM_ERR_ARG;   // ascending, disjoint
+      prev_end = pi.first + pi.n;
+      uint64_t n_elems = 0;
+      int rc = tm_shard_validate(plan->descs.data() + pi.first, pi.n, r, D, &pi.e, &n_elems);
+      if (rc != TM_OK) return rc;
+      rc = tm_bounds_u128(n_elems, r, D, &pi.lo, &pi.hi);
+      if (rc != TM_OK) return rc;
+      if (out_elems != nullptr) out_elems[p] = pi.hi - pi.lo;
+    }
+    const tms::WorkspaceLayout l = tms::workspace_layout(plan->work.segs.size(), plan->work.n_items(), true);
+    if (workspace_needed != nullptr) *workspace_needed = l.total;
+    if (d_workspace == nullptr && d_outs == nullptr) return TM_OK;   // size query
     if (d_outs == nullptr || out_capacities == nullptr) return TM_ERR_ARG;
     if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+    if (d_workspace != nullptr && workspace_bytes < l.total) return TM_ERR_CAPACITY;
+    std::vector<std::pair<uint64_t, uint64_t>> outs;
     for (uint32_t p = 0; p < n_planes; ++p) {
       const uint64_t bytes = (planes[p].hi - planes[p].lo) * planes[p].e;
       if (bytes == 0) continue;
@@ -301,210 +392,69 @@ int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const
       if (((uintptr_t)d_outs[p] & 1) != 0) return TM_ERR_ALIGN;
       if (out_capacities[p] < bytes) return TM_ERR_CAPACITY;
       const uint64_t o = (uint64_t)(uintptr_t)d_outs[p];
-      for (const tm_desc& d : plan->descs)
-        if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, o, bytes)) return TM_ERR_OVERLAP;
+      if (plan_overlaps(plan, o, bytes)) return TM_ERR_OVERLAP;
       for (const auto& q : outs)
-        if (ranges_overlap(o, bytes, q.first, q.second)) return TM_ERR_OVERLAP;
+        if (tms::ranges_overlap(o, bytes, q.first, q.second)) return TM_ERR_OVERLAP;
       outs.emplace_back(o, bytes);
-      base = std::min(base, o);
     }
-  }
-  if (base == ~0ull) base = 0;
-  // one pass over the descriptors: the pack pieces of tensor k, then the emit pieces that read tensor k
-  tms::WorkList wl;
-  tms::WorkListBuilder builder(&wl);
-  size_t cursor = 0;            // next pack piece of the plan
-  uint32_t p = 0;               // current plane
-  uint64_t start = 0;           // element index, inside plane p, of tensor k's first element
-  for (uint64_t k = 0; k < n_desc; ++k) {
-    uint64_t seen = 0;
-    while (seen < plan->descs[k].nbytes) {
-      const tms::Seg& s = plan->work.segs[cursor++];
-      builder.add(s);
-      seen += s.nbytes;
-    }
-    while (p < n_planes && k >= planes[p].first + planes[p].n) { ++p; start = 0; }
-    if (p < n_planes && k >= planes[p].first) {
-      const PlaneInfo& pi = planes[p];
-      const uint64_t count = plan->descs[k].nbytes / pi.e;
-      const uint64_t a = std::max(pi.lo, start), b = std::min(pi.hi, start + count);
-      if (a < b) {
-        const uint64_t out = dry ? (uint64_t)256 * (a - pi.lo) : (uint64_t)(uintptr_t)d_outs[p] + (a - pi.lo) * pi.e;
-        tm_shard_append(&builder, &plan->descs[k], 1, pi.e, a - start, b - start, out, dry ? 0 : base, 0xffffffffu);
+    // for every descriptor inside a plane: its plane and the plane-wide index of its first element
+    std::vector<int32_t> desc_plane(n_desc, -1);
+    std::vector<uint64_t> desc_start(n_desc, 0);
+    for (uint32_t p = 0; p < n_planes; ++p) {
+      uint64_t start = 0;
+      for (uint64_t k = planes[p].first; k < planes[p].first + planes[p].n; ++k) {
+        desc_plane[k] = (int32_t)p;
+        desc_start[k] = start;
+        start += plan->descs[k].nbytes / planes[p].e;
       }
-      start += count;
     }
-  }
-  builder.finish();
-  const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size() + 2 * n_desc + 8, wl.n_items() + 2 * n_desc + 8);
-  if (workspace_needed != nullptr) *workspace_needed = l.total;
-  if (dry) return TM_OK;
-  const tms::WorkspaceLayout exact = tms::workspace_layout(wl.segs.size(), wl.n_items());
-  if (workspace_bytes < exact.total) return TM_ERR_CAPACITY;
-  int rc = upload_worklist(wl, exact, (uint8_t*)d_workspace, (cudaStream_t)stream);
-  if (rc != TM_OK) return rc;
-  plan->emit_work = std::move(wl);
-  plan->emit_layout = exact;
-  plan->d_emit_workspace = (uint8_t*)d_workspace;
-  plan->emit_base = base;
-  plan->emit_outs = std::move(outs);
-  return TM_OK;
+    // one emit record per piece: the piece's bytes that are shard elements, and where they go
+    std::vector<tms::Emit> emits(plan->work.segs.size());
+    for (size_t i = 0; i < emits.size(); ++i) {
+      tms::Emit& em = emits[i];
+      em.out = 0;
+      em.begin = 0;
+      em.len = 0;
+      const uint32_t k = plan->piece_desc[i];
+      if (desc_plane[k] < 0) continue;
+      const PlaneInfo& pi = planes[desc_plane[k]];
+      const uint64_t start = desc_start[k], count = plan->descs[k].nbytes / pi.e;
+      const uint64_t a = std::max(pi.lo, start), b = std::min(pi.hi, start + count);
+      if (a >= b) continue;
+      const tms::Seg& s = plan->work.segs[i];
+      const uint64_t x = s.tensor - (uint64_t)(uintptr_t)plan->descs[k].ptr;   // piece = tensor bytes [x, x + nbytes)
+      const uint64_t sa = (a - start) * pi.e, sb = (b - start) * pi.e;         // shard = tensor bytes [sa, sb)
+      const uint64_t lo = std::max(x, sa), hi = std::min(x + s.nbytes, sb);
+      if (lo >= hi) continue;
+      em.begin = (uint32_t)(lo - x);
+      em.len = (uint32_t)(hi - lo);
+      em.out = (uint64_t)(uintptr_t)d_outs[desc_plane[k]] + ((start * pi.e + lo) - pi.lo * pi.e);   // plane byte - shard's first byte
+    }
+    if (d_workspace != nullptr) {   // without a workspace the records are only computed, for inspection on the host
+      int rc = tms::upload_worklist(plan->work, &emits, l, (uint8_t*)d_workspace, stream);
+      if (rc != TM_OK) return rc;
+    }
+    plan->emits = std::move(emits);
+    plan->emit_layout = l;
+    plan->d_emit_workspace = (uint8_t*)d_workspace;
+    plan->emit_outs = std::move(outs);
+    return TM_OK;
+  });
 }
 
 int tm_state_pack_emit(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint64_t* d_checksums,
                        void* stream) {
-  if (plan == nullptr || d_buckets == nullptr) return TM_ERR_ARG;
+  int rc = check_buckets(plan, d_buckets, capacity, d_checksums);
+  if (rc != TM_OK) return rc;
   if (plan->d_emit_workspace == nullptr) return TM_ERR_STATE;
-  if (((uintptr_t)d_buckets & 255) != 0 || ((uintptr_t)d_checksums & 7) != 0) return TM_ERR_ALIGN;
-  if (capacity < plan->total_bytes) return TM_ERR_CAPACITY;
-  const uint64_t base = (uint64_t)(uintptr_t)d_buckets;
-  for (const tm_desc& d : plan->descs)
-    if (ranges_overlap((uint64_t)(uintptr_t)d.ptr, d.nbytes, base, plan->total_bytes)) return TM_ERR_OVERLAP;
   for (const auto& o : plan->emit_outs)
-    if (ranges_overlap(o.first, o.second, base, plan->total_bytes)) return TM_ERR_OVERLAP;
-  cudaStream_t st = (cudaStream_t)stream;
+    if (tms::ranges_overlap(o.first, o.second, (uint64_t)(uintptr_t)d_buckets, plan->total_bytes)) return TM_ERR_OVERLAP;
   if (d_checksums != nullptr)
-    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), st));
-  const uint8_t* ws = plan->d_emit_workspace;
-  int e = tms::launch_pack_emit_ring((const tms::Seg*)(ws + plan->emit_layout.segs_off),
-                                     (const uint32_t*)(ws + plan->emit_layout.items_off),
-                                     (uint32_t)plan->emit_work.n_items(), (uint8_t*)d_buckets,
-                                     (unsigned long long*)d_checksums, (uint8_t*)(uintptr_t)plan->emit_base,
-                                     (int*)plan->d_emit_workspace, stream);
-  return e == 0 ? TM_OK : cuda_fail(e);
-}
-
-int tm_shard_bounds(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi) {
-  if (lo == nullptr || hi == nullptr) return TM_ERR_ARG;
-  return tm_bounds_u128(n_elems, r, D, lo, hi);
-}
-
-int tm_shard_workspace(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
-                       uint64_t* workspace_bytes) {
-  if (workspace_bytes == nullptr) return TM_ERR_ARG;
-  uint32_t e = 0;
-  uint64_t n_elems = 0;
-  int rc = tm_shard_validate(plane_descs, n_desc, r, D, &e, &n_elems);
-  if (rc != TM_OK) return rc;
-  uint64_t lo = 0, hi = 0;
-  rc = tm_bounds_u128(n_elems, r, D, &lo, &hi);
-  if (rc != TM_OK) return rc;
-  // upper bound on pieces: every tensor adds at most two partial pieces to the chunk count
-  const uint64_t chunk = tms::tuning().shard_chunk_bytes;
-  const uint64_t max_segs = (hi - lo) * e / chunk + 2 * n_desc + 2;
-  *workspace_bytes = tms::workspace_layout(max_segs, max_segs).total;
-  return TM_OK;
-}
-
-// Shared body of shard extract (tensors -> flat) and shard insert (flat -> tensors).
-static int shard_run(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, void* d_flat,
-                     uint64_t flat_capacity, uint64_t* elems, void* d_workspace, uint64_t workspace_bytes,
-                     void* stream, bool to_tensors) {
-  uint32_t e = 0;
-  uint64_t n_elems = 0;
-  int rc = tm_shard_validate(plane_descs, n_desc, r, D, &e, &n_elems);
-  if (rc != TM_OK) return rc;
-  uint64_t lo = 0, hi = 0;
-  rc = tm_bounds_u128(n_elems, r, D, &lo, &hi);
-  if (rc != TM_OK) return rc;
-  if (elems != nullptr) *elems = hi - lo;
-  if (hi == lo) return TM_OK;
-  if (d_flat == nullptr || d_workspace == nullptr) return TM_ERR_ARG;
-  if (((uintptr_t)d_flat & 1) != 0 || ((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
-  const uint64_t flat_bytes = (hi - lo) * e;
-  if (flat_capacity < flat_bytes) return TM_ERR_CAPACITY;
-  const uint64_t flat_addr = (uint64_t)(uintptr_t)d_flat;
-  for (uint64_t k = 0; k < n_desc; ++k)
-    if (ranges_overlap((uint64_t)(uintptr_t)plane_descs[k].ptr, plane_descs[k].nbytes, flat_addr, flat_bytes))
-      return TM_ERR_OVERLAP;
-  tms::WorkList wl;
-  tm_shard_worklist(plane_descs, n_desc, e, lo, hi, flat_addr, &wl);
-  const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
-  if (workspace_bytes < l.total) return TM_ERR_CAPACITY;
-  rc = upload_worklist(wl, l, (uint8_t*)d_workspace, (cudaStream_t)stream);
-  if (rc != TM_OK) return rc;
-  const uint8_t* ws = (const uint8_t*)d_workspace;
-  auto copy_fn = tms::tuning().use_ring ? tms::launch_copy_ring : tms::launch_copy;
-  int err = copy_fn((const tms::Seg*)(ws + l.segs_off), (const uint32_t*)(ws + l.items_off),
-                    (uint32_t)wl.n_items(), (uint8_t*)d_flat, to_tensors, (int*)d_workspace, stream);
-  return err == 0 ? TM_OK : cuda_fail(err);
-}
-
-int tm_shard_extract(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, void* d_out,
-                     uint64_t out_capacity, uint64_t* out_elems, void* d_workspace,
-                     uint64_t workspace_bytes, void* stream) {
-  return shard_run(plane_descs, n_desc, r, D, d_out, out_capacity, out_elems, d_workspace, workspace_bytes,
-                   stream, /*to_tensors=*/false);
-}
-
-int tm_shard_extract_planes(const tm_desc* descs, const uint64_t* plane_n_desc, uint32_t n_planes, uint32_t r,
-                            uint32_t D, void* const* d_outs, const uint64_t* out_capacities,
-                            uint64_t* out_elems, void* d_workspace, uint64_t workspace_bytes, void* stream) {
-  if (descs == nullptr || plane_n_desc == nullptr || n_planes == 0 || d_outs == nullptr ||
-      out_capacities == nullptr)
-    return TM_ERR_ARG;
-  if (d_workspace == nullptr) return TM_ERR_ARG;
-  if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
-  struct PlaneInfo { const tm_desc* d; uint64_t n; uint32_t e; uint64_t lo, hi; };
-  std::vector<PlaneInfo> planes(n_planes);
-  const tm_desc* cursor = descs;
-  uint64_t base = ~0ull;
-  for (uint32_t p = 0; p < n_planes; ++p) {
-    PlaneInfo& pi = planes[p];
-    pi.d = cursor;
-    pi.n = plane_n_desc[p];
-    uint64_t n_elems = 0;
-    int rc = tm_shard_validate(pi.d, pi.n, r, D, &pi.e, &n_elems);
-    if (rc != TM_OK) return rc;
-    rc = tm_bounds_u128(n_elems, r, D, &pi.lo, &pi.hi);
-    if (rc != TM_OK) return rc;
-    cursor += pi.n;
-    if (pi.hi == pi.lo) continue;
-    if (d_outs[p] == nullptr) return TM_ERR_ARG;
-    if (((uintptr_t)d_outs[p] & 1) != 0) return TM_ERR_ALIGN;
-    if (out_capacities[p] < (pi.hi - pi.lo) * pi.e) return TM_ERR_CAPACITY;
-    base = std::min(base, (uint64_t)(uintptr_t)d_outs[p]);
-  }
-  // no output may overlap a tensor of any plane, nor another output
-  const uint64_t n_total = (uint64_t)(cursor - descs);
-  for (uint32_t p = 0; p < n_planes; ++p) {
-    if (planes[p].hi == planes[p].lo) continue;
-    const uint64_t o = (uint64_t)(uintptr_t)d_outs[p], ob = (planes[p].hi - planes[p].lo) * planes[p].e;
-    for (uint64_t k = 0; k < n_total; ++k)
-      if (ranges_overlap((uint64_t)(uintptr_t)descs[k].ptr, descs[k].nbytes, o, ob)) return TM_ERR_OVERLAP;
-    for (uint32_t q = p + 1; q < n_planes; ++q) {
-      if (planes[q].hi == planes[q].lo) continue;
-      if (ranges_overlap(o, ob, (uint64_t)(uintptr_t)d_outs[q], (planes[q].hi - planes[q].lo) * planes[q].e))
-        return TM_ERR_OVERLAP;
-    }
-  }
-  if (out_elems != nullptr)
-    for (uint32_t p = 0; p < n_planes; ++p) out_elems[p] = planes[p].hi - planes[p].lo;
-  if (base == ~0ull) return TM_OK;   // every shard is empty
-  tms::WorkList wl;
-  tms::WorkListBuilder builder(&wl);
-  for (uint32_t p = 0; p < n_planes; ++p)
-    if (planes[p].hi != planes[p].lo)
-      tm_shard_append(&builder, planes[p].d, planes[p].n, planes[p].e, planes[p].lo, planes[p].hi,
-                      (uint64_t)(uintptr_t)d_outs[p], base, 0);
-  builder.finish();
-  const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
-  if (workspace_bytes < l.total) return TM_ERR_CAPACITY;
-  int rc = upload_worklist(wl, l, (uint8_t*)d_workspace, (cudaStream_t)stream);
-  if (rc != TM_OK) return rc;
-  const uint8_t* ws = (const uint8_t*)d_workspace;
-  auto copy_fn = tms::tuning().use_ring ? tms::launch_copy_ring : tms::launch_copy;
-  int err = copy_fn((const tms::Seg*)(ws + l.segs_off), (const uint32_t*)(ws + l.items_off),
-                    (uint32_t)wl.n_items(), (uint8_t*)(uintptr_t)base, /*to_tensors=*/false,
-                    (int*)d_workspace, stream);
-  return err == 0 ? TM_OK : cuda_fail(err);
-}
-
-int tm_shard_insert(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, const void* d_in,
-                    uint64_t in_bytes, uint64_t* in_elems, void* d_workspace, uint64_t workspace_bytes,
-                    void* stream) {
-  return shard_run(plane_descs, n_desc, r, D, const_cast<void*>(d_in), in_bytes, in_elems, d_workspace,
-                   workspace_bytes, stream, /*to_tensors=*/true);
+    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), (cudaStream_t)stream));
+  tms::RingLaunch a = ring_args(plan, plan->d_emit_workspace, plan->emit_layout, d_buckets, d_checksums);
+  a.d_emits = (const tms::Emit*)(plan->d_emit_workspace + plan->emit_layout.emits_off);
+  int e = tms::launch_ring(tms::kRingPackEmit, a, stream);
+  return e == 0 ? TM_OK : tms::cuda_fail(e);
 }
 
 int tm_selftest_bounded_wait(void* d_workspace, uint64_t limit_ns, void* stream) {
@@ -512,11 +462,11 @@ int tm_selftest_bounded_wait(void* d_workspace, uint64_t limit_ns, void* stream)
   if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
   TM_CUDA(cudaMemsetAsync(d_workspace, 0, tms::kStatusBlockBytes, (cudaStream_t)stream));
   int e = tms::launch_wait_selftest((int*)d_workspace, limit_ns, stream);
-  return e == 0 ? TM_OK : cuda_fail(e);
+  return e == 0 ? TM_OK : tms::cuda_fail(e);
 }
 
 int tm_workspace_status(const void* d_workspace, void* stream, int* device_status) {
-  return read_status(d_workspace, (cudaStream_t)stream, device_status);
+  return tms::read_status_word(d_workspace, stream, device_status);
 }
 
 int tm_checksum(const void* d_bytes, uint64_t nbytes, uint64_t bucket_bytes, uint64_t* d_checksums,
@@ -530,8 +480,8 @@ int tm_checksum(const void* d_bytes, uint64_t nbytes, uint64_t bucket_bytes, uin
   cudaStream_t st = (cudaStream_t)stream;
   TM_CUDA(cudaMemsetAsync(d_checksums, 0, n_buckets * sizeof(uint64_t), st));
   int e = tms::launch_checksum((const uint8_t*)d_bytes, nbytes, bucket_bytes,
-                              (unsigned long long*)d_checksums, stream);
-  return e == 0 ? TM_OK : cuda_fail(e);
+                              (unsigned long long*)d_checksums, tms::tuning(), stream);
+  return e == 0 ? TM_OK : tms::cuda_fail(e);
 }
 
 const char* tm_strerror(int status) {
@@ -546,6 +496,8 @@ const char* tm_strerror(int status) {
     case TM_ERR_CUDA: return "CUDA runtime error";
     case TM_ERR_TIMEOUT: return "bounded device wait expired";
     case TM_ERR_STATE: return "plan has no uploaded work list";
+    case TM_ERR_VERIFY: return "checksum mismatch after the last transfer round";
+    case TM_ERR_TRANSPORT: return "transport callback failed";
     default: return "unknown status";
   }
 }

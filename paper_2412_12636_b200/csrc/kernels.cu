@@ -1,17 +1,15 @@
 // Register-path kernels of the role-state mover for sm_100a: the stand-alone checksum
-// (checksum_kernel, the one every tm_checksum call runs), and pack_kernel / copy_kernel — the
-// load/store versions of pack, unpack and shard copy.  The main path of pack, unpack and shard
-// extract is the bulk-copy ring in ring_kernels.cu; pack_kernel / copy_kernel run when
-// TM_USE_RING=0 is set (for A/B measurement) and copy_kernel serves tm_shard_extract_static.
+// (checksum_kernel, the one every tm_checksum call runs) and copy_to_flat_kernel, a load/store
+// gather of pieces into a flat buffer that serves tm_shard_extract_static.  Pack, unpack and the
+// other shard calls run on the bulk-copy ring in ring_kernels.cu.
 // Everything here is HBM-bound byte movement with one 64-bit multiply-add per 8 bytes; there is no
 // contraction, so no tensor cores.
 //
-// Work distribution: a persistent grid walks the item list with a grid stride.  An item with one
-// piece is copied by the whole block; an item with several small pieces gives one warp per piece.
-// All global accesses of the main loops are 16-byte vectors, consecutive lanes on consecutive
-// vectors.  A piece whose tensor address is not 16-byte aligned is read as aligned vectors and
-// re-aligned in registers (funnel shifts), so stores and checksum words stay aligned to the flat
-// buffer.
+// Work distribution: a persistent grid walks the item or tile list with a grid stride.  An item with
+// one piece is copied by the whole block; an item with several small pieces gives one warp per
+// piece.  All global accesses of the main loops are 16-byte vectors, consecutive lanes on
+// consecutive vectors.  A piece whose tensor address is not 16-byte aligned is read as aligned
+// vectors and re-aligned in registers (funnel shifts), so stores stay aligned to the flat buffer.
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -39,37 +37,8 @@ __device__ __forceinline__ void block_flush(u64 value, u64* target, u64* smem) {
 }
 
 __global__ void __launch_bounds__(kThreads, kMinBlocks)
-pack_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
-            uint8_t* __restrict__ stream, u64* __restrict__ checksums) {
-  __shared__ u64 red[kWarps];
-  Cksum ck;
-  u64 total = 0;            // this thread's share of the checksum of bucket `cur`
-  uint32_t cur = 0xffffffffu;
-  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const uint32_t first = item_first[item], last = item_first[item + 1];
-    const uint32_t bucket = segs[first].bucket;
-    if (bucket != cur) {    // uniform over the block
-      if (cur != 0xffffffffu && checksums != nullptr) block_flush(total, checksums + cur, red);
-      total = 0;
-      cur = bucket;
-    }
-    // one piece: the whole block copies it; several pieces: one warp per piece
-    const bool single = (last - first == 1);
-    const uint32_t g = single ? threadIdx.x : lane, G = single ? kThreads : 32u;
-    for (uint32_t i = first + (single ? 0u : warp); i < last; i += (single ? 1u : (uint32_t)kWarps)) {
-      const Seg s = segs[i];
-      pack_piece(s, stream, g, G, ck);
-      total += ck.finish(s.word0);
-    }
-  }
-  if (cur != 0xffffffffu && checksums != nullptr) block_flush(total, checksums + cur, red);
-}
-
-template <bool TO_TENSORS>
-__global__ void __launch_bounds__(kThreads, kMinBlocks)
-copy_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
-            uint8_t* __restrict__ flat) {
+copy_to_flat_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
+                    uint8_t* __restrict__ flat) {
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t first = item_first[item], last = item_first[item + 1];
@@ -77,9 +46,7 @@ copy_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
     const uint32_t g = single ? threadIdx.x : lane, G = single ? kThreads : 32u;
     for (uint32_t i = first + (single ? 0u : warp); i < last; i += (single ? 1u : (uint32_t)kWarps)) {
       const Seg s = segs[i];
-      uint8_t* t = reinterpret_cast<uint8_t*>(s.tensor);
-      uint8_t* f = flat + s.off;
-      copy_piece(TO_TENSORS ? t : f, TO_TENSORS ? f : t, s.nbytes, g, G);
+      copy_piece(flat + s.off, reinterpret_cast<const uint8_t*>(s.tensor), s.nbytes, g, G);
     }
   }
 }
@@ -163,49 +130,35 @@ int device_sm_count(int* sms) {
   return 0;
 }
 
-static int grid_for(uint64_t n_items, uint32_t* grid) {
+static int grid_for(uint64_t n_items, uint32_t ctas_per_sm, uint32_t* grid) {
   int sms = 0;
   int rc = device_sm_count(&sms);
   if (rc != 0) return rc;
-  uint64_t g = (uint64_t)sms * tuning().ctas_per_sm;
+  uint64_t g = (uint64_t)sms * (ctas_per_sm == 0 ? 1u : ctas_per_sm);
   if (g > n_items) g = n_items;
   if (g == 0) g = 1;
   *grid = (uint32_t)g;
   return 0;
 }
 
-int launch_pack(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                unsigned long long* d_checksums, int* /*d_status*/, void* stream) {
+int launch_copy_to_flat(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
+                        uint32_t ctas_per_sm, void* stream) {
   uint32_t grid = 0;
-  int rc = grid_for(n_items, &grid);
+  int rc = grid_for(n_items, ctas_per_sm, &grid);
   if (rc != 0) return rc;
-  pack_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_stream,
-                                                          d_checksums);
-  count_launch();
-  return (int)cudaGetLastError();
-}
-
-int launch_copy(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
-                bool to_tensors, int* /*d_status*/, void* stream) {
-  uint32_t grid = 0;
-  int rc = grid_for(n_items, &grid);
-  if (rc != 0) return rc;
-  if (to_tensors)
-    copy_kernel<true><<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat);
-  else
-    copy_kernel<false><<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat);
+  copy_to_flat_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat);
   count_launch();
   return (int)cudaGetLastError();
 }
 
 int launch_checksum(const uint8_t* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
-                    unsigned long long* d_checksums, void* stream) {
+                    unsigned long long* d_checksums, const Tuning& t, void* stream) {
   const uint64_t n_buckets = (nbytes + bucket_bytes - 1) / bucket_bytes;
-  const uint32_t tile = (uint32_t)tuning().cksum_tile_bytes;
+  const uint32_t tile = (uint32_t)t.cksum_tile_bytes;
   const uint64_t tpb = (bucket_bytes + tile - 1) / tile;
   const uint64_t n_tiles = n_buckets * tpb;
   uint32_t grid = 0;
-  int rc = grid_for(n_tiles, &grid);
+  int rc = grid_for(n_tiles, t.ctas_per_sm, &grid);
   if (rc != 0) return rc;
   checksum_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(d_bytes, nbytes, bucket_bytes, (uint32_t)tpb,
                                                               n_tiles, tile, d_checksums);

@@ -17,6 +17,11 @@
 //
 // Small pieces (items that group several pieces, or single pieces below kBulkMinVectors) are
 // copied by the consumer warps with the register routines of device_util.cuh.
+//
+// Pack-and-emit: a pack piece may carry a second destination for a sub-range of its bytes (the part
+// of the tensor that falls into a distributed-optimizer shard).  The consumer warps write that
+// sub-range to the shard output from the same shared-memory stage that feeds the stream and the
+// checksum, so the tensor is read from HBM once for all three results.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -34,8 +39,7 @@ constexpr int kConsWarps = 8;
 constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kRingThreads = kConsThreads + 64;     // + one producer warp + one store warp
 constexpr uint32_t kBulkMinVectors = 128;           // pieces below 2 KiB are not worth a stage
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-constexpr uint32_t kEmitBucket = 0xffffffffu;       // marks an emit piece in a pack-and-emit list
+constexpr unsigned long long kDrainLimitNs = 2000000000ull;   // bound of the producer's final wait for its own loads
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
@@ -61,9 +65,9 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Waits for the phase with the given parity; gives up after kWaitLimitNs or when the block aborts.
+// Waits for the phase with the given parity; gives up after limit_ns or when the block aborts.
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag,
-                                          unsigned long long limit_ns = kWaitLimitNs) {
+                                          unsigned long long limit_ns) {
   if (mbar_try(b, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
@@ -151,18 +155,52 @@ __device__ __forceinline__ void consumer_flush(u64 value, u64* target) {
   if ((threadIdx.x & 31) == 0 && value != 0) atomicAdd(target, value);
 }
 
+// Copies n bytes (even) from shared memory `s` to global memory `d`, both at any even alignment, with
+// threads c, c + C, ...: 2-byte copies up to the first 16-byte boundary of the destination, aligned
+// 16-byte stores re-aligned from two aligned shared-memory vectors, 2-byte copies for the tail.
+// Reads at most one aligned 16-byte vector past the last source byte (inside the stage's slack).
+__device__ __forceinline__ void smem_to_global(uint8_t* d, const uint8_t* s, uint32_t n, uint32_t c, uint32_t C) {
+  uint32_t head = (uint32_t)((0 - (uintptr_t)d) & 15);
+  if (head > n) head = n;
+  if (2 * c < head) st2(d + 2 * c, (uint32_t)(*reinterpret_cast<const uint16_t*>(s + 2 * c)));
+  d += head;
+  s += head;
+  n -= head;
+  const uint32_t nfull = n >> 4, rem = n & 15;
+  const uint32_t a = smem_u32(s) & 15;
+  const uint4* sa = reinterpret_cast<const uint4*>(s - a);
+  if (a == 0) {
+    for (uint32_t v = c; v < nfull; v += C) st16(d + (size_t)v * 16u, sa[v]);
+  } else {
+    const uint32_t ws = a >> 2, bs = (a & 3) * 8;
+    for (uint32_t v = c; v < nfull; v += C) st16(d + (size_t)v * 16u, shift_pair(sa[v], sa[v + 1], ws, bs));
+  }
+  const size_t tl = (size_t)nfull * 16u;
+  const uint32_t gt = C - 1 - c;
+  if (2 * gt < rem) st2(d + tl + 2 * gt, (uint32_t)(*reinterpret_cast<const uint16_t*>(s + tl + 2 * gt)));
+}
+
+// Emits the part of piece bytes [lo, hi) (hi - lo <= 16) that lies inside the emit span, straight
+// from the tensor: the few bytes of a bulk piece that do not travel through the ring.
+__device__ __forceinline__ void emit_direct(const Emit& em, const uint8_t* piece_src, uint32_t lo, uint32_t hi,
+                                            uint32_t c) {
+  const uint32_t b = lo > em.begin ? lo : em.begin;
+  const uint32_t e = hi < em.begin + em.len ? hi : em.begin + em.len;
+  if (b + 2 * c < e) st2(reinterpret_cast<uint8_t*>(em.out) + (b - em.begin) + 2 * c, ld2(piece_src + b + 2 * c));
+}
+
 // PACK: tensors -> stream with padding and checksums.  Otherwise a plain copy of pieces, direction
 // given by TO_TENSORS (PACK implies TO_TENSORS == false).  VERIFY (with TO_TENSORS): the unpack also
 // accumulates the per-bucket checksums of the stream it reads — data and padding bytes as they
 // arrived — so that a receiver checks and scatters in one pass over the buckets.
-// EMIT (with PACK): the list also holds "emit" pieces, marked by bucket == kEmitBucket, which are
-// plain copies tensor -> flat2 (a shard output); they sit next to the pack pieces that read the same
-// tensor bytes, so their source is served from the L2 rather than read from DRAM a second time.
+// EMIT (with PACK): emits[i] gives piece i an optional second destination for a sub-range of its
+// bytes; the consumers write it from the stage in shared memory (bulk pieces) or re-read the few KiB
+// of a small piece they have just copied (served by L1 / L2).
 template <bool PACK, bool TO_TENSORS, bool VERIFY, bool EMIT>
 __global__ void __launch_bounds__(kRingThreads, 1)
 ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
             uint8_t* __restrict__ flat, u64* __restrict__ checksums, int* __restrict__ status,
-            uint8_t* __restrict__ flat2) {
+            const Emit* __restrict__ emits, unsigned long long wait_limit_ns) {
   extern __shared__ __align__(128) uint8_t ring[];
   __shared__ RingShared sh;
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -187,10 +225,10 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       if (item_first[item + 1] - first != 1) continue;
       const Seg s = segs[first];
       BulkPlan p;
-      if (!plan_bulk<TO_TENSORS>(s, (EMIT && s.bucket == kEmitBucket) ? flat2 : flat, p)) continue;
+      if (!plan_bulk<TO_TENSORS>(s, flat, p)) continue;
       const uint32_t extra = p.a != 0 ? 1u : 0u;
       for (uint32_t t = 0; t < p.ntiles; ++t) {
-        if (!mbar_wait(&sh.empty[stage], phase ^ 1u, abort_flag)) {
+        if (!mbar_wait(&sh.empty[stage], phase ^ 1u, abort_flag, wait_limit_ns)) {
           raise_timeout(status, &sh);
           ok = false;
           break;
@@ -204,15 +242,19 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
         if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok || *abort_flag != 0) {
-      // leave no copy in flight: the latest load of each stage must have landed before the block exits
+    // Leave no copy in flight, whatever the other roles do: the newest load of every stage must have
+    // landed before this thread — and with it possibly the block — exits.  try_wait only observes the
+    // phase, so the consumers' own waits on the same barriers are not disturbed.  The bound here is a
+    // constant of its own; a shortened wait_limit_ns does not shorten it.
+    {
       uint32_t n = issued < (uint32_t)kRingStages ? issued : (uint32_t)kRingStages;
       uint32_t st = stage, ph = phase;
       for (uint32_t k = 0; k < n; ++k) {
         if (st == 0) { st = kRingStages; ph ^= 1u; }
         --st;
+        if (mbar_try(&sh.full[st], ph)) continue;
         const unsigned long long t0 = global_ns();
-        while (!mbar_try(&sh.full[st], ph) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try(&sh.full[st], ph) && global_ns() - t0 < kDrainLimitNs) {}
       }
     }
     return;
@@ -229,9 +271,9 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       if (item_first[item + 1] - first != 1) continue;
       const Seg s = segs[first];
       BulkPlan p;
-      if (!plan_bulk<TO_TENSORS>(s, (EMIT && s.bucket == kEmitBucket) ? flat2 : flat, p)) continue;
+      if (!plan_bulk<TO_TENSORS>(s, flat, p)) continue;
       for (uint32_t t = 0; t < p.ntiles; ++t) {
-        if (!mbar_wait(&sh.full[stage], phase, abort_flag)) {
+        if (!mbar_wait(&sh.full[stage], phase, abort_flag, wait_limit_ns)) {
           raise_timeout(status, &sh);
           ok = false;
           break;
@@ -272,10 +314,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
   bool ok = true;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t first = item_first[item], last = item_first[item + 1];
-    const bool emit_item = EMIT && segs[first].bucket == kEmitBucket;   // uniform over the block
-    const bool packing = PACK && !emit_item;
-    uint8_t* const base = emit_item ? flat2 : flat;
-    if ((PACK || VERIFY) && !emit_item) {
+    if (PACK || VERIFY) {
       const uint32_t bucket = segs[first].bucket;
       if (bucket != cur) {   // uniform over the consumers
         if (cur != 0xffffffffu && checksums != nullptr) consumer_flush(total, checksums + cur);
@@ -289,19 +328,25 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
     bool bulk = false;
     if (single) {
       s0 = segs[first];
-      bulk = plan_bulk<TO_TENSORS>(s0, base, p);
+      bulk = plan_bulk<TO_TENSORS>(s0, flat, p);
     }
     if (!bulk) {
       if (!ok) continue;
       const uint32_t g = single ? c : lane, G = single ? (uint32_t)kConsThreads : 32u;
       for (uint32_t i = first + (single ? 0u : warp); i < last; i += (single ? 1u : (uint32_t)kConsWarps)) {
         const Seg s = segs[i];
-        if (packing) {
+        if (PACK) {
           pack_piece(s, flat, g, G, ck);
           total += ck.finish(s.word0);
+          if (EMIT) {
+            const Emit em = emits[i];
+            if (em.len != 0)
+              copy_piece(reinterpret_cast<uint8_t*>(em.out), reinterpret_cast<const uint8_t*>(s.tensor) + em.begin,
+                         em.len, g, G);
+          }
         } else {
           uint8_t* t = reinterpret_cast<uint8_t*>(s.tensor);
-          uint8_t* f = base + s.off;
+          uint8_t* f = flat + s.off;
           copy_piece(TO_TENSORS ? t : f, TO_TENSORS ? f : t, s.nbytes, g, G);
           if (VERIFY) {   // the piece's span of the stream, padding included, in aligned vectors
             const uint32_t nvec = (s.nbytes + s.pad) >> 4;
@@ -316,22 +361,33 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
     if (!ok) continue;
     // bulk piece: head bytes directly, full vectors through the ring, tail (and padding) directly
     if (2 * c < p.head) st2(p.dst - p.head + 2 * c, ld2(p.src - p.head + 2 * c));
+    Emit em;
+    em.out = 0; em.begin = 0; em.len = 0;
+    if (EMIT) {
+      em = emits[first];
+      if (em.len != 0) {   // piece bytes outside the ring's share: before the first and after the last full vector
+        const uint8_t* piece_src = p.src - p.head;
+        if (p.head != 0) emit_direct(em, piece_src, 0, p.head, c);
+        if (p.rem != 0) emit_direct(em, piece_src, p.head + p.nfull * 16u, s0.nbytes, c);
+      }
+    }
     const uint32_t ws = p.a >> 2, bs = (p.a & 3) * 8;
     for (uint32_t t = 0; t < p.ntiles; ++t) {
       // the vote keeps the warp together: either all of its lanes go on or none does
-      if (!__all_sync(0xffffffffu, mbar_wait(&sh.full[stage], phase, abort_flag))) {
+      if (!__all_sync(0xffffffffu, mbar_wait(&sh.full[stage], phase, abort_flag, wait_limit_ns))) {
         raise_timeout(status, &sh);
         ok = false;
         break;
       }
       uint32_t cnt = p.nfull - t * p.V;
       if (cnt > p.V) cnt = p.V;
-      const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageStride);
+      const uint8_t* stage_base = ring + (size_t)stage * kStageStride;
+      const uint4* sp = reinterpret_cast<const uint4*>(stage_base);
       const uint32_t vbase = t * p.V;
       uint8_t* d = p.dst + (size_t)vbase * 16u;
       // VERIFY: the stream piece starts 256-byte aligned, so stage vector v is stream vector vbase + v
       if (p.straight) {
-        if (packing || VERIFY) {   // the store thread moves the data; only the checksum is left to do
+        if (PACK || VERIFY) {   // the store thread moves the data; only the checksum is left to do
 #pragma unroll 4
           for (uint32_t v = c; v < cnt; v += kConsThreads) ck.add(sp[v], vbase + v);
         }
@@ -341,16 +397,25 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
           const uint4 lo = sp[v];
           const uint4 x = shift_pair(lo, sp[v + 1], ws, bs);
           st16(d + (size_t)v * 16u, x);
-          if (packing) ck.add(x, vbase + v);
+          if (PACK) ck.add(x, vbase + v);
           if (VERIFY) ck.add(lo, vbase + v);
         }
+      }
+      if (EMIT && em.len != 0) {
+        // this stage holds piece bytes [s_lo, s_hi), byte b at stage_base + a + (b - s_lo)
+        const uint32_t s_lo = p.head + vbase * 16u, s_hi = s_lo + cnt * 16u;
+        const uint32_t b = s_lo > em.begin ? s_lo : em.begin;
+        const uint32_t e = s_hi < em.begin + em.len ? s_hi : em.begin + em.len;
+        if (b < e)
+          smem_to_global(reinterpret_cast<uint8_t*>(em.out) + (b - em.begin), stage_base + p.a + (b - s_lo), e - b, c,
+                         (uint32_t)kConsThreads);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.empty[stage]);
       if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
     }
     if (!ok) continue;
-    if (packing) {
+    if (PACK) {
       // the vector with the tensor's last (n mod 16) bytes, then whole vectors of zero padding
       const uint32_t nvec = (s0.nbytes + s0.pad) >> 4;
       for (uint32_t v = p.nfull + c; v < nvec; v += kConsThreads) {
@@ -402,47 +467,50 @@ int launch_wait_selftest(int* d_status, unsigned long long limit_ns, void* strea
   return (int)cudaGetLastError();
 }
 
+constexpr int kMaxDevices = 64;
+
+// The ring needs more dynamic shared memory than the default limit; the attribute is set once per
+// kernel and device.
 template <typename K>
-static int launch_ring(K kernel, const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
-                       unsigned long long* d_checksums, int* d_status, void* stream, uint8_t* d_flat2 = nullptr) {
+static cudaError_t ensure_smem(K kernel, size_t smem, int dev, bool* done) {
+  if (dev >= 0 && dev < kMaxDevices && done[dev]) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess && dev >= 0 && dev < kMaxDevices) done[dev] = true;
+  return e;
+}
+
+template <bool PACK, bool TO_TENSORS, bool VERIFY, bool EMIT>
+static int launch_ring_t(const RingLaunch& a, void* stream) {
+  static bool attr_done[kMaxDevices] = {false};
   int sms = 0;
   int rc = device_sm_count(&sms);
   if (rc != 0) return rc;
-  const size_t smem = (size_t)kRingStages * kStageStride;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return (int)e;
-  uint64_t grid = (uint64_t)sms * tuning().ring_ctas_per_sm;
-  if (grid > n_items) grid = n_items;
+  const size_t smem = (size_t)kRingStages * kStageStride;
+  auto kernel = ring_kernel<PACK, TO_TENSORS, VERIFY, EMIT>;
+  e = ensure_smem(kernel, smem, dev, attr_done);
+  if (e != cudaSuccess) return (int)e;
+  uint64_t grid = (uint64_t)sms * (a.ctas_per_sm == 0 ? 1u : a.ctas_per_sm);
+  if (grid > a.n_items) grid = a.n_items;
   if (grid == 0) grid = 1;
-  kernel<<<(uint32_t)grid, kRingThreads, smem, (cudaStream_t)stream>>>(d_segs, d_item_first, n_items, d_flat,
-                                                                    d_checksums, d_status, d_flat2);
+  kernel<<<(uint32_t)grid, kRingThreads, smem, (cudaStream_t)stream>>>(a.d_segs, a.d_item_first, a.n_items, a.d_flat,
+                                                                    a.d_checksums, a.d_status, a.d_emits,
+                                                                    a.wait_limit_ns);
   count_launch();
   return (int)cudaGetLastError();
 }
 
-int launch_pack_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                     unsigned long long* d_checksums, int* d_status, void* stream) {
-  return launch_ring(ring_kernel<true, false, false, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
-                     stream);
-}
-
-int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
-                     bool to_tensors, int* d_status, void* stream) {
-  if (to_tensors)
-    return launch_ring(ring_kernel<false, true, false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
-  return launch_ring(ring_kernel<false, false, false, false>, d_segs, d_item_first, n_items, d_flat, nullptr, d_status, stream);
-}
-
-int launch_unpack_verify_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                              unsigned long long* d_checksums, int* d_status, void* stream) {
-  return launch_ring(ring_kernel<false, true, true, false>, d_segs, d_item_first, n_items, d_stream, d_checksums, d_status,
-                     stream);
-}
-
-int launch_pack_emit_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                          unsigned long long* d_checksums, uint8_t* d_emit_base, int* d_status, void* stream) {
-  return launch_ring(ring_kernel<true, false, false, true>, d_segs, d_item_first, n_items, d_stream, d_checksums,
-                     d_status, stream, d_emit_base);
+int launch_ring(RingMode mode, const RingLaunch& a, void* stream) {
+  switch (mode) {
+    case kRingPack: return launch_ring_t<true, false, false, false>(a, stream);
+    case kRingPackEmit: return launch_ring_t<true, false, false, true>(a, stream);
+    case kRingToFlat: return launch_ring_t<false, false, false, false>(a, stream);
+    case kRingToTensors: return launch_ring_t<false, true, false, false>(a, stream);
+    case kRingToTensorsVerify: return launch_ring_t<false, true, true, false>(a, stream);
+  }
+  return (int)cudaErrorInvalidValue;
 }
 
 }  // namespace tms

@@ -13,21 +13,20 @@
 //   * a request whose work list does not fit is refused with TM_ERR_CAPACITY, nothing is launched;
 //   * all calls on one GPU share the one array and it still holds the previous call's list, so the
 //     status block is cleared on every call and two calls whose device work may overlap (different
-//     streams, or one stream per thread) would overwrite each other's list: issue them on one stream;
+//     streams) would overwrite each other's list: issue them on one stream;
+//   * the host side of a call — clear, two list copies, launch — runs under one lock, so threads that
+//     share a stream cannot interleave their sequences;
+//   * the list is copied from ordinary (pageable) host memory: the call returns once the stream has
+//     taken the copies, which may mean waiting for earlier work in that stream;
 //   * the first call on each GPU looks up the array's device address (cudaGetSymbolAddress) with that
 //     GPU current; make that first call outside any stream capture.
 // No cudaMalloc, cudaFree or other allocating routine is called here.
 #include <cuda_runtime.h>
 
 #include <mutex>
+#include <new>
 
 #include "tm_internal.h"
-
-int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
-int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_t D,
-                      uint32_t* elem_size, uint64_t* n_elems);
-void tm_shard_worklist(const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo, uint64_t hi,
-                       uint64_t d_out, tms::WorkList* wl);
 
 // In host code this name is only a handle for the runtime, not a device address: never pass it to a
 // kernel.  The address comes from cudaGetSymbolAddress below.
@@ -39,13 +38,13 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
 uint8_t* g_scratch_addr[kMaxDevices] = {nullptr};
 
-// Device address of the scratch array on the current device; looked up once per device.
+// Device address of the scratch array on the current device; looked up once per device.  The caller
+// holds g_mutex.
 cudaError_t scratch_for_current_device(uint8_t** out) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  std::lock_guard<std::mutex> lock(g_mutex);
   if (g_scratch_addr[dev] == nullptr) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_static_scratch);
@@ -58,9 +57,8 @@ cudaError_t scratch_for_current_device(uint8_t** out) {
 
 }  // namespace
 
-extern "C" int tm_shard_extract_static(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
-                                       void* d_out, uint64_t out_capacity, uint64_t* out_elems,
-                                       void* stream) {
+static int extract_static(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D, void* d_out,
+                          uint64_t out_capacity, uint64_t* out_elems, void* stream) {
   uint32_t e = 0;
   uint64_t n_elems = 0;
   int rc = tm_shard_validate(plane_descs, n_desc, r, D, &e, &n_elems);
@@ -75,31 +73,45 @@ extern "C" int tm_shard_extract_static(const tm_desc* plane_descs, uint64_t n_de
   const uint64_t out_bytes = (hi - lo) * e;
   if (out_capacity < out_bytes) return TM_ERR_CAPACITY;
   // refuse oversized requests from the byte count alone, before building any list
-  const uint64_t chunk = tms::tuning().shard_chunk_bytes;
-  const uint64_t min_segs = out_bytes / chunk;
+  const tms::Tuning opt = tms::tuning();
+  const uint64_t min_segs = out_bytes / opt.shard_chunk_bytes;
   if (tms::workspace_layout(min_segs, 1).total > TM_STATIC_SCRATCH_BYTES) return TM_ERR_CAPACITY;
   const uint64_t out_addr = (uint64_t)(uintptr_t)d_out;
-  for (uint64_t k = 0; k < n_desc; ++k) {
-    const uint64_t a = (uint64_t)(uintptr_t)plane_descs[k].ptr;
-    if (a < out_addr + out_bytes && out_addr < a + plane_descs[k].nbytes) return TM_ERR_OVERLAP;
-  }
+  for (uint64_t k = 0; k < n_desc; ++k)
+    if (tms::ranges_overlap((uint64_t)(uintptr_t)plane_descs[k].ptr, plane_descs[k].nbytes, out_addr, out_bytes))
+      return TM_ERR_OVERLAP;
   tms::WorkList wl;
-  tm_shard_worklist(plane_descs, n_desc, e, lo, hi, out_addr, &wl);
+  tm_shard_worklist(opt, plane_descs, n_desc, e, lo, hi, out_addr, &wl);
   const tms::WorkspaceLayout l = tms::workspace_layout(wl.segs.size(), wl.n_items());
   if (l.total > TM_STATIC_SCRATCH_BYTES) return TM_ERR_CAPACITY;
 
+  // One lock around the address lookup and the whole clear / copy / copy / launch sequence: two threads
+  // that issue on the same stream cannot interleave, so each kernel reads the list its own call wrote.
+  std::lock_guard<std::mutex> lock(g_mutex);
   uint8_t* scratch = nullptr;
   cudaError_t ce = scratch_for_current_device(&scratch);
-  if (ce != cudaSuccess) return TM_ERR_CUDA;
+  if (ce != cudaSuccess) return tms::cuda_fail((int)ce);
   cudaStream_t st = (cudaStream_t)stream;
   // the array still holds the previous call's status block and list: clear the former, overwrite the latter
-  if ((ce = cudaMemsetAsync(scratch, 0, tms::kStatusBlockBytes, st)) != cudaSuccess) return TM_ERR_CUDA;
+  if ((ce = cudaMemsetAsync(scratch, 0, tms::kStatusBlockBytes, st)) != cudaSuccess) return tms::cuda_fail((int)ce);
   if ((ce = cudaMemcpyAsync(scratch + l.segs_off, wl.segs.data(), wl.segs.size() * sizeof(tms::Seg),
-                            cudaMemcpyHostToDevice, st)) != cudaSuccess) return TM_ERR_CUDA;
+                            cudaMemcpyHostToDevice, st)) != cudaSuccess) return tms::cuda_fail((int)ce);
   if ((ce = cudaMemcpyAsync(scratch + l.items_off, wl.item_first.data(), wl.item_first.size() * sizeof(uint32_t),
-                            cudaMemcpyHostToDevice, st)) != cudaSuccess) return TM_ERR_CUDA;
-  const int err = tms::launch_copy((const tms::Seg*)(scratch + l.segs_off), (const uint32_t*)(scratch + l.items_off),
-                                   (uint32_t)wl.n_items(), (uint8_t*)d_out, /*to_tensors=*/false,
-                                   (int*)scratch, stream);
-  return err == 0 ? TM_OK : TM_ERR_CUDA;
+                            cudaMemcpyHostToDevice, st)) != cudaSuccess) return tms::cuda_fail((int)ce);
+  const int err = tms::launch_copy_to_flat((const tms::Seg*)(scratch + l.segs_off),
+                                           (const uint32_t*)(scratch + l.items_off), (uint32_t)wl.n_items(),
+                                           (uint8_t*)d_out, opt.ctas_per_sm, stream);
+  return err == 0 ? TM_OK : tms::cuda_fail(err);
+}
+
+extern "C" int tm_shard_extract_static(const tm_desc* plane_descs, uint64_t n_desc, uint32_t r, uint32_t D,
+                                       void* d_out, uint64_t out_capacity, uint64_t* out_elems,
+                                       void* stream) {
+  try {
+    return extract_static(plane_descs, n_desc, r, D, d_out, out_capacity, out_elems, stream);
+  } catch (const std::bad_alloc&) {
+    return TM_ERR_CAPACITY;
+  } catch (...) {
+    return TM_ERR_ARG;
+  }
 }

@@ -22,6 +22,15 @@ struct alignas(16) Seg {
 };
 static_assert(sizeof(Seg) == 32, "Seg is 32 bytes on host and device");
 
+// Optional second destination of a pack piece: bytes [begin, begin + len) of the piece also go to
+// the device address `out` (a shard output).  len == 0: nothing to emit.  One record per piece.
+struct alignas(16) Emit {
+  uint64_t out;
+  uint32_t begin;
+  uint32_t len;
+};
+static_assert(sizeof(Emit) == 16, "Emit is 16 bytes on host and device");
+
 // A work list: pieces grouped into items.  Item i owns pieces [item_first[i], item_first[i+1]).
 // A large piece is an item of its own (a whole thread block works on it); runs of small pieces
 // share an item (one warp per piece).  All pieces of an item lie in one bucket.
@@ -31,15 +40,22 @@ struct WorkList {
   uint64_t n_items() const { return item_first.empty() ? 0 : item_first.size() - 1; }
 };
 
+// Process-wide tuning values (tm_options_get / tm_options_set); a plan keeps the copy it was built with.
+typedef tm_options Tuning;
+Tuning tuning();
+Tuning default_tuning();
+int set_tuning(const Tuning* t);   // validates; nullptr restores the defaults
+
 // Incrementally groups pieces into items.
 class WorkListBuilder {
  public:
-  explicit WorkListBuilder(WorkList* wl);
+  WorkListBuilder(WorkList* wl, const Tuning& t);
   void add(const Seg& s);
   void finish();
 
  private:
   WorkList* wl_;
+  Tuning t_;
   uint64_t group_bytes_ = 0;
   uint32_t group_count_ = 0;
   uint32_t group_bucket_ = 0;
@@ -47,71 +63,124 @@ class WorkListBuilder {
   void close_group();
 };
 
-struct Tuning {
-  uint64_t chunk_bytes;    // largest piece of a pack / unpack plan; multiple of 256
-  uint64_t shard_chunk_bytes;  // largest piece of a shard list (smaller: a shard is a fraction of a role)
-  uint64_t small_bytes;    // pieces below this share items
-  uint64_t group_bytes;    // byte budget of a shared item
-  uint32_t group_max;      // piece budget of a shared item
-  uint64_t cksum_tile_bytes;   // tile of the stand-alone checksum kernel; multiple of 256
-  uint32_t ctas_per_sm;    // persistent grid = SMs * ctas_per_sm (register-path kernels)
-  uint32_t ring_ctas_per_sm;  // same for the bulk-copy ring kernels (96 KiB of shared memory each)
-  bool use_ring;           // pack / unpack / shard through the bulk-copy ring kernels
-};
-const Tuning& tuning();
-
 // Byte layout of a work list inside a device workspace.
 struct WorkspaceLayout {
   uint64_t segs_off;    // 256: after the status block
   uint64_t items_off;
+  uint64_t emits_off;   // one Emit per piece (only lists that emit; otherwise == total)
   uint64_t total;
 };
-WorkspaceLayout workspace_layout(uint64_t n_segs, uint64_t n_items);
+WorkspaceLayout workspace_layout(uint64_t n_segs, uint64_t n_items, bool with_emits = false);
 constexpr uint64_t kStatusBlockBytes = 256;  // word 0: device status (0 ok, else tm_status)
 
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+inline bool ranges_overlap(uint64_t a, uint64_t an, uint64_t b, uint64_t bn) { return a < b + bn && b < a + an; }
 
-// ---- kernel launchers (kernels.cu).  Each returns a cudaError_t as int. -----------------------
-int launch_pack(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                unsigned long long* d_checksums, int* d_status, void* stream);
-// flat -> tensors when to_tensors, tensors -> flat otherwise (no checksum, no padding)
-int launch_copy(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
-                bool to_tensors, int* d_status, void* stream);
-// bulk-copy ring versions (ring_kernels.cu); d_status receives TM_ERR_TIMEOUT if a bounded wait expires
-int launch_pack_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                     unsigned long long* d_checksums, int* d_status, void* stream);
-int launch_copy_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
-                     bool to_tensors, int* d_status, void* stream);
-int launch_unpack_verify_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                              unsigned long long* d_checksums, int* d_status, void* stream);
-int launch_pack_emit_ring(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_stream,
-                          unsigned long long* d_checksums, uint8_t* d_emit_base, int* d_status, void* stream);
+// Sizes beyond these are refused: with them no sum of sizes or offsets formed by the planner can
+// reach 2^63.
+constexpr uint64_t kMaxTensorBytes = 1ull << 46;
+constexpr uint64_t kMaxDescs = 1ull << 24;
+constexpr uint64_t kMaxTotalBytes = 1ull << 56;
+
+// ---- kernel launchers.  Each returns a cudaError_t as int. -----------------------------------
+// What a ring launch does with the pieces of its list.
+enum RingMode {
+  kRingPack,          // tensors -> stream, zero padding, per-bucket checksums
+  kRingPackEmit,      // the same, and every piece's emit span also goes to its shard output
+  kRingToFlat,        // tensors -> flat buffer (shard extract)
+  kRingToTensors,     // flat buffer -> tensors (unpack, shard insert)
+  kRingToTensorsVerify  // unpack that also accumulates the checksums of the stream as read
+};
+struct RingLaunch {
+  const Seg* d_segs = nullptr;
+  const uint32_t* d_item_first = nullptr;
+  const Emit* d_emits = nullptr;
+  uint32_t n_items = 0;
+  uint8_t* d_flat = nullptr;
+  unsigned long long* d_checksums = nullptr;
+  int* d_status = nullptr;
+  unsigned long long wait_limit_ns = 0;
+  uint32_t ctas_per_sm = 1;
+};
+int launch_ring(RingMode mode, const RingLaunch& a, void* stream);
+// register-path copy tensors -> flat (used by the entry point that owns its scratch)
+int launch_copy_to_flat(const Seg* d_segs, const uint32_t* d_item_first, uint32_t n_items, uint8_t* d_flat,
+                        uint32_t ctas_per_sm, void* stream);
 int launch_wait_selftest(int* d_status, unsigned long long limit_ns, void* stream);
 int launch_checksum(const uint8_t* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
-                    unsigned long long* d_checksums, void* stream);
+                    unsigned long long* d_checksums, const Tuning& t, void* stream);
 int device_sm_count(int* sms);
 void count_launch();
 
+// ---- shared host helpers (api.cpp) ------------------------------------------------------------
+int cuda_fail(int cuda_error);   // records the error for tm_last_cuda_error(), returns TM_ERR_CUDA
+// Uploads status block + pieces + items (+ emits) as one image; asynchronous on `stream`.
+int upload_worklist(const WorkList& wl, const std::vector<Emit>* emits, const WorkspaceLayout& l, uint8_t* d_ws,
+                    void* stream);
+int read_status_word(const void* d_ws, void* stream, int* device_status);
+
 }  // namespace tms
+
+// One part of a tensor that a plan touches (a range plan touches only part of the role).
+struct tm_part {
+  uint64_t addr;
+  uint64_t nbytes;
+};
 
 struct tm_plan {
   std::vector<tm_desc> descs;
-  std::vector<uint64_t> offsets;
+  std::vector<uint64_t> offsets;     // off_k in the complete stream
+  tms::Tuning opt{};
   uint64_t bucket_bytes = 0;
-  uint64_t total_bytes = 0;
-  uint64_t n_buckets = 0;
+  uint64_t whole_bytes = 0;          // T of the complete stream
+  uint64_t whole_buckets = 0;
+  uint64_t first_bucket = 0;         // range plans: first bucket covered
+  uint64_t range_begin = 0;          // = first_bucket * bucket_bytes
+  uint64_t total_bytes = 0;          // bytes this plan packs / unpacks (the whole stream, or the range)
+  uint64_t n_buckets = 0;            // buckets this plan covers
   tms::WorkList work;
+  std::vector<uint32_t> piece_desc;  // descriptor index of every piece
+  std::vector<tm_part> parts;        // tensor parts touched by the plan
+  uint64_t box_lo = 0, box_hi = 0;   // address bounding box of `parts`
   tms::WorkspaceLayout ws_layout{};
   // set by tm_plan_upload
   uint8_t* d_workspace = nullptr;
-  // set by tm_plan_attach_shards: pack pieces interleaved with the emit pieces of the attached shards
-  tms::WorkList emit_work;
+  // set by tm_plan_attach_shards: the same work list with one emit record per piece
+  std::vector<tms::Emit> emits;
   tms::WorkspaceLayout emit_layout{};
   uint8_t* d_emit_workspace = nullptr;
-  uint64_t emit_base = 0;                      // lowest shard output address; emit offsets are relative to it
   std::vector<std::pair<uint64_t, uint64_t>> emit_outs;   // (address, bytes) of every non-empty shard output
   // lazily computed: 0 unknown, 1 targets disjoint, -1 targets overlap
   mutable int targets_disjoint = 0;
 };
+
+// Reusable shard plan: the same [lo, hi) of one or several planes, bound to flat buffers.
+struct tm_shard_plan {
+  std::vector<tm_desc> descs;
+  std::vector<uint64_t> plane_n;
+  std::vector<uint32_t> elem_size;
+  std::vector<uint64_t> lo, hi;
+  tms::Tuning opt{};
+  uint32_t r = 0, D = 0;
+  // set by tm_shard_plan_bind
+  tms::WorkList work;
+  tms::WorkspaceLayout layout{};
+  std::vector<std::pair<uint64_t, uint64_t>> flats;   // (address, bytes) per plane (0 bytes: empty shard)
+  uint64_t base = 0;                                   // lowest flat address; piece offsets are relative to it
+  uint8_t* d_workspace = nullptr;
+  int targets_disjoint = 0;
+};
+
+// planner (plan.cpp)
+int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, bool ranged,
+                  uint64_t first_bucket, uint64_t n_buckets);
+int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
+int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_t D, uint32_t* elem_size,
+                      uint64_t* n_elems);
+void tm_shard_append(tms::WorkListBuilder* builder, const tms::Tuning& t, const tm_desc* descs, uint64_t n_desc,
+                     uint32_t e, uint64_t lo, uint64_t hi, uint64_t d_out, uint64_t flat_base);
+void tm_shard_worklist(const tms::Tuning& t, const tm_desc* descs, uint64_t n_desc, uint32_t e, uint64_t lo,
+                       uint64_t hi, uint64_t d_out, tms::WorkList* wl);
+int tm_parts_disjoint(std::vector<tm_part> parts);   // 1 disjoint, -1 overlap
 
 #endif  // TM_INTERNAL_H

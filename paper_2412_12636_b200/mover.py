@@ -17,9 +17,10 @@ class RoleMover:
     """A packed-stream plan for one role's tensors with its uploaded work list."""
 
     def __init__(self, descs: Sequence[Tuple[int, int, int, int]], bucket_bytes: int, device="cuda",
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, first_bucket: Optional[int] = None,
+                 n_buckets: Optional[int] = None):
         self.device = torch.device(device)
-        self.plan = binding.Plan(descs, bucket_bytes)
+        self.plan = binding.Plan(descs, bucket_bytes, first_bucket, n_buckets)
         self._elem_sizes = [d[2] for d in descs]
         self.total_bytes = self.plan.total_bytes
         self.n_buckets = self.plan.n_buckets
@@ -40,14 +41,16 @@ class RoleMover:
                               None if checksums is None else checksums.data_ptr(), _stream_handle(stream))
 
     def attach_shards(self, planes: Sequence[Tuple[int, int]], r: int, D: int,
-                      stream: Optional[torch.cuda.Stream] = None):
+                      stream: Optional[torch.cuda.Stream] = None, outs: Optional[Sequence[torch.Tensor]] = None):
         """Prepares pack_emit: `planes` = (first descriptor, count) runs of this role's descriptors.
-        Allocates and returns the shard output buffers (one uint8 tensor per plane)."""
+        Returns the shard output buffers (one uint8 tensor per plane): `outs` if given (range plans of
+        one role share them), freshly allocated otherwise."""
         elems, need = binding.tm_plan_attach_shards(self.plan, planes, r, D, None, None, None, 0, 0)
         sizes = []
         for (first, count), n in zip(planes, elems):
             sizes.append(n * self._elem_sizes[first])
-        self.emit_outs = [torch.empty(max(n, 1), dtype=torch.uint8, device=self.device)[:n] for n in sizes]
+        self.emit_outs = list(outs) if outs is not None else \
+            [torch.empty(max(n, 1), dtype=torch.uint8, device=self.device)[:n] for n in sizes]
         self.emit_workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         binding.tm_plan_attach_shards(self.plan, planes, r, D, [o.data_ptr() for o in self.emit_outs], sizes,
                                       self.emit_workspace.data_ptr(), need, _stream_handle(stream))
@@ -79,7 +82,8 @@ class RoleMover:
 
 
 class ShardExtractor:
-    """Shard r of D of one plane (tensors of one element size), with its scratch workspace."""
+    """Shard r of D of one plane (tensors of one element size) through the one-shot calls, which
+    build and upload the work list on every call; owns the scratch workspace they need."""
 
     def __init__(self, plane_descs: Sequence[Tuple[int, int, int, int]], r: int, D: int, device="cuda"):
         self.device = torch.device(device)
@@ -108,7 +112,8 @@ class ShardExtractor:
 
 
 class MultiShardExtractor:
-    """Shard r of D of several planes (each with its own element size) in one launch."""
+    """Shard r of D of several planes (each with its own element size) in one launch, through the
+    one-shot call tm_shard_extract_planes."""
 
     def __init__(self, planes: Sequence[Sequence[Tuple[int, int, int, int]]], r: int, D: int, device="cuda"):
         import ctypes
@@ -141,48 +146,104 @@ class MultiShardExtractor:
         return list(self._got)
 
 
-class WaveMover:
-    """The same role cut into waves of whole buckets (see waves.py), one plan per wave.
+class ShardPlanMover:
+    """Shard r of D of several planes as a reusable plan (tm_shard_plan_*): the work list is built and
+    uploaded once, bound to flat buffers that this object owns (or is given); extract and insert are
+    then one kernel launch each with no host work."""
 
-    Wave i packs into stream bytes [begin_i, end_i) and produces the checksums of its own buckets,
-    so waves can be packed one after another — into slices of one full-size buffer, or into a
-    small ring of staging slots when the packed copy must not take a second role's worth of memory
-    (the paper's §8.5 rule: the transfer channel is a bounded, recycled buffer).  The concatenation
-    of the waves' streams and checksum lists equals what a single plan produces."""
+    def __init__(self, planes: Sequence[Sequence[Tuple[int, int, int, int]]], r: int, D: int, device="cuda",
+                 flats: Optional[Sequence[torch.Tensor]] = None, stream: Optional[torch.cuda.Stream] = None):
+        self.device = torch.device(device)
+        self.plan = binding.ShardPlan(planes, r, D)
+        self.out_bytes = self.plan.out_bytes
+        self.workspace = torch.empty(max(self.plan.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
+        self.flats = list(flats) if flats is not None else \
+            [torch.empty(n, dtype=torch.uint8, device=self.device) for n in self.out_bytes]
+        self.rebind(self.flats, stream)
+
+    def rebind(self, flats: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
+        self.flats = list(flats)
+        self.plan.bind([f.data_ptr() for f in self.flats], [f.numel() * f.element_size() for f in self.flats],
+                       self.workspace.data_ptr(), self.workspace.numel(), _stream_handle(stream))
+
+    def extract(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        self.plan.extract(_stream_handle(stream))
+
+    def insert(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        self.plan.insert(_stream_handle(stream))
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        return self.plan.status(_stream_handle(stream))
+
+
+class WaveMover:
+    """The same role cut into waves of whole buckets, one range plan (tm_plan_create_range) per wave.
+
+    Wave i packs stream bytes [begin_i, end_i) and produces the checksums of its own buckets, so
+    waves can be packed one after another — into slices of one full-size buffer, or into a small
+    ring of staging slots when the packed copy must not take a second role's worth of memory (the
+    paper's §8.5 rule: the transfer channel is a bounded, recycled buffer).  The concatenation of the
+    waves' streams and checksum lists equals what a single plan produces."""
 
     def __init__(self, descs: Sequence[Tuple[int, int, int, int]], bucket_bytes: int, wave_bytes: int,
                  device="cuda", stream: Optional[torch.cuda.Stream] = None):
-        from . import waves as _waves
-        whole = binding.Plan(descs, bucket_bytes)
-        self.total_bytes, self.n_buckets, self.bucket_bytes = whole.total_bytes, whole.n_buckets, bucket_bytes
-        offsets = whole.offsets()
-        whole.close()
-        sizes = [d[1] for d in descs]
-        self.waves = _waves.cut_waves(sizes, offsets, self.total_bytes, bucket_bytes, wave_bytes)
+        per_wave = max(1, wave_bytes // bucket_bytes)
+        arr = binding.make_descs(descs)
         self.movers = []
-        self.tensor_ranges = []   # per wave: (first tensor, last tensor + 1) touched by the wave
-        for w in self.waves:
-            part_descs = [(descs[p.tensor][0] + p.byte_start, p.nbytes, descs[p.tensor][2], descs[p.tensor][3])
-                          for p in w.parts]
-            self.movers.append(RoleMover(part_descs, bucket_bytes, device, stream))
-            self.tensor_ranges.append((w.parts[0].tensor, w.parts[-1].tensor + 1))
+        first = 0
+        while True:
+            m = RoleMover.__new__(RoleMover)
+            m.device = torch.device(device)
+            m.plan = binding.Plan(arr, bucket_bytes, first, per_wave)
+            m._elem_sizes = [d[2] for d in descs]
+            m.total_bytes, m.n_buckets, m.bucket_bytes = m.plan.total_bytes, m.plan.n_buckets, bucket_bytes
+            m.workspace = torch.empty(m.plan.workspace_bytes, dtype=torch.uint8, device=m.device)
+            m.plan.upload(m.workspace.data_ptr(), m.workspace.numel(), _stream_handle(stream))
+            self.movers.append(m)
+            first += per_wave
+            if first >= m.plan.whole_buckets:
+                break
+        p0 = self.movers[0].plan
+        self.total_bytes, self.n_buckets, self.bucket_bytes = p0.whole_bytes, p0.whole_buckets, bucket_bytes
+        self.n_waves = len(self.movers)
+        # tensors touched by each wave, from the stream offsets the planner reports
+        offsets = p0.offsets()
+        self.tensor_ranges = []
+        k = 0
+        for m in self.movers:
+            lo, hi = m.plan.stream_begin, m.plan.stream_begin + m.plan.total_bytes
+            while k < len(descs) and offsets[k] + descs[k][1] <= lo:
+                k += 1
+            j = k
+            while j < len(descs) and offsets[j] < hi:
+                j += 1
+            self.tensor_ranges.append((k, j))
+
+    def wave_span(self, i: int) -> Tuple[int, int]:
+        """(stream_begin, stream_end) of wave i in the complete stream."""
+        p = self.movers[i].plan
+        return p.stream_begin, p.stream_begin + p.total_bytes
+
+    def wave_buckets(self, i: int) -> Tuple[int, int]:
+        """(first bucket, bucket count) of wave i."""
+        p = self.movers[i].plan
+        return p.first_bucket, p.n_buckets
 
     def wave_bytes(self, i: int) -> int:
-        return self.waves[i].stream_end - self.waves[i].stream_begin
+        return self.movers[i].plan.total_bytes
 
     def pack_wave_into(self, i: int, slot: torch.Tensor, checksums: Optional[torch.Tensor],
                        stream: Optional[torch.cuda.Stream] = None) -> int:
         """Packs wave i into a staging slot (any 256-byte-aligned buffer of at least wave_bytes(i)
         bytes) — the bounded-channel mode: the caller ships the slot and reuses it for a later wave.
         `checksums` is the full per-bucket array of the role.  Returns the bytes written."""
-        w = self.waves[i]
-        cks = None if checksums is None else checksums[w.first_bucket:w.first_bucket + w.n_buckets]
+        first, count = self.wave_buckets(i)
+        cks = None if checksums is None else checksums[first:first + count]
         self.movers[i].pack(slot, cks, stream)
-        return w.stream_end - w.stream_begin
+        return self.wave_bytes(i)
 
     def pack_wave(self, i: int, buckets: torch.Tensor, checksums: Optional[torch.Tensor],
                   stream: Optional[torch.cuda.Stream] = None) -> None:
         """Packs wave i into its slice of the full-size `buckets` / `checksums` tensors."""
-        w = self.waves[i]
-        cks = None if checksums is None else checksums[w.first_bucket:w.first_bucket + w.n_buckets]
-        self.movers[i].pack(buckets[w.stream_begin:w.stream_end], cks, stream)
+        begin, end = self.wave_span(i)
+        self.pack_wave_into(i, buckets[begin:end], checksums, stream)

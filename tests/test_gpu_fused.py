@@ -1,0 +1,229 @@
+"""GPU parity of the fused and reusable forms: pack that emits the shards from the same staged copy
+(whole plans and range plans), reusable shard plans, buckets that live in pinned host memory, and
+the kernels' bounded waits made to expire.  Everything is compared with the CPU oracle bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_12636_b200 import binding, layouts
+from paper_2412_12636_b200.mover import RoleMover, ShardPlanMover, WaveMover
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _cuda():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.load_library()
+    torch.cuda.set_device(0)
+    yield
+
+
+def _adversarial_by_elem_size(n, max_log2, seed):
+    specs = sorted(layouts.adversarial_specs(n, max_log2=max_log2), key=lambda s: s.elem_size)
+    state = layouts.materialize_adversarial(specs, "cuda", seed=seed)
+    runs, k = [], 0
+    for e in (2, 4, 8):
+        c = sum(1 for s in specs if s.elem_size == e)
+        runs.append((k, c))
+        k += c
+    return state, runs
+
+
+def _expected_shards(oracle, host, state, planes, r, D):
+    out = []
+    for first, count in planes:
+        sub = host[first:first + count]
+        out.append(oracle.shard(sub, [h.size for h in sub], state.specs[first].elem_size, r, D))
+    return out
+
+
+@pytest.mark.parametrize("case", ["cfg0-r1of2", "cfg0-r2of3-small-buckets", "adv-r5of7", "adv-r63of64", "adv-D>N"])
+def test_range_plans_pack_emit_through_a_slot_ring(oracle_mod, case):
+    """The role travels as runs of whole buckets through two recycled slots; every run's launch also
+    writes its part of the three shards.  Stream, checksums and shards must equal the oracle's."""
+    if case.startswith("cfg0"):
+        cfg = layouts.role_config(0)
+        state = layouts.materialize(cfg, "cuda")
+        P = len(cfg.model)
+        planes = [(P, P), (2 * P, P), (3 * P, P)]
+        r, D, B, per = (1, 2, cfg.bucket_bytes, 3) if case == "cfg0-r1of2" else (2, 3, 256 * 1024, 7)
+    else:
+        state, planes = _adversarial_by_elem_size(700, 18, seed=13)
+        r, D = {"adv-r5of7": (5, 7), "adv-r63of64": (63, 64), "adv-D>N": (10 ** 9 - 1, 10 ** 9)}[case]
+        B, per = 1 << 20, 5
+    host = G.host_tensors(state)
+    exp_stream, exp_cks = oracle_mod.pack(host, B)
+    exp_shards = _expected_shards(oracle_mod, host, state, planes, r, D)
+    descs = state.descs()
+    outs = [G.guarded(e.size) for e in exp_shards]
+    slots = [G.guarded(per * B) for _ in range(2)]
+    cks = torch.zeros(exp_cks.size, dtype=torch.int64, device="cuda")
+    received = torch.empty(exp_stream.size, dtype=torch.uint8, device="cuda")
+    first, i = 0, 0
+    while first < exp_cks.size:
+        m = RoleMover(descs, B, first_bucket=first, n_buckets=per)
+        got = m.attach_shards(planes, r, D, outs=[o[1] for o in outs])
+        assert [g.numel() for g in got] == [e.size for e in exp_shards]
+        whole, slot = slots[i % 2]
+        slot.fill_(0x77)
+        launches = binding.tm_launch_count()
+        m.pack_emit(slot, cks[first:first + m.n_buckets])
+        torch.cuda.synchronize()
+        assert binding.tm_launch_count() == launches + 1 and m.status() == 0
+        assert G.guards_intact(whole, per * B) and bool((slot[m.total_bytes:] == 0x77).all())
+        lo = m.plan.stream_begin
+        received[lo:lo + m.total_bytes].copy_(slot[:m.total_bytes])
+        first += per
+        i += 1
+    assert np.array_equal(received.cpu().numpy(), exp_stream)
+    assert np.array_equal(G.u64(cks), exp_cks)
+    for (whole, out), e in zip(outs, exp_shards):
+        assert np.array_equal(out.cpu().numpy(), e), G._first_diff(out.cpu().numpy(), e)
+        assert G.guards_intact(whole, e.size)
+
+
+@pytest.mark.parametrize("misalign", [0, 2, 6, 10])
+def test_pack_emit_every_output_alignment(oracle_mod, misalign):
+    # one bulk tensor, shard boundaries mid-stage; shard output at every 2-byte-granular alignment class
+    n = 3 * 32768 + 4100
+    arena = torch.randint(0, 256, (4 * n + 64,), dtype=torch.uint8, device="cuda",
+                          generator=torch.Generator("cuda").manual_seed(misalign + 1))
+    for src_mis in (0, 4):
+        t = arena[src_mis:src_mis + 4 * n]
+        spec = layouts.TensorSpec("t", n, torch.float32, 1, 0)
+        state = layouts.RoleState("one", [spec], [t], 1 << 20, 0, 1, arena)
+        host = G.host_tensors(state)
+        exp_stream, exp_cks = oracle_mod.pack(host, 1 << 20)
+        for r, D in ((0, 1), (1, 3), (6, 7)):
+            expect = oracle_mod.shard(host, [4 * n], 4, r, D)
+            m = RoleMover(state.descs(), 1 << 20)
+            whole, out = G.guarded(expect.size + 16)
+            out = out[misalign:misalign + expect.size]
+            m.attach_shards([(0, 1)], r, D, outs=[out])
+            wb, buckets = G.guarded(m.total_bytes)
+            cks = m.alloc_checksums()
+            m.pack_emit(buckets, cks)
+            torch.cuda.synchronize()
+            assert m.status() == 0
+            assert np.array_equal(buckets.cpu().numpy(), exp_stream) and np.array_equal(G.u64(cks), exp_cks)
+            assert np.array_equal(out.cpu().numpy(), expect), (src_mis, r, D, G._first_diff(out.cpu().numpy(), expect))
+            assert bool((whole[:G.GUARD + misalign] == G.GUARD_BYTE).all())
+            assert bool((whole[G.GUARD + misalign + expect.size:] == G.GUARD_BYTE).all())
+            assert G.guards_intact(wb, m.total_bytes)
+
+
+def test_shard_plan_extract_and_insert_match_the_oracle(oracle_mod):
+    cfg = layouts.role_config(0)
+    st0 = layouts.materialize(cfg, "cuda")
+    adv = layouts.materialize_adversarial(layouts.adversarial_specs(400, max_log2=17), "cuda", seed=31)
+    cases = [
+        (st0, [st0.plane_indices(p) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)], 1, 2),
+        (adv, [adv.elem_size_indices(e) for e in (4, 2, 8)], 17, 64),
+        (adv, [adv.elem_size_indices(e) for e in (8, 4)], 10 ** 9 - 1, 10 ** 9),    # one-element shards
+        (adv, [adv.elem_size_indices(e) for e in (8, 4)], 0, 10 ** 9),              # empty shards: no launch
+    ]
+    for st, planes, r, D in cases:
+        plane_descs = [st.descs_of(idx) for idx in planes]
+        host = [[st.host_bytes(i) for i in idx] for idx in planes]
+        expect = [oracle_mod.shard(h, [x.size for x in h], st.specs[idx[0]].elem_size, r, D)
+                  for h, idx in zip(host, planes)]
+        bufs = [G.guarded(e.size + 16) for e in expect]
+        flats = [b[1][2 * p:2 * p + e.size] for p, (b, e) in enumerate(zip(bufs, expect))]   # 2-byte-granular outputs
+        sp = ShardPlanMover(plane_descs, r, D, flats=flats)
+        assert sp.out_bytes == [e.size for e in expect]
+        launches = binding.tm_launch_count()
+        for _ in range(3):                                   # reuse: no host work between launches
+            sp.extract()
+        torch.cuda.synchronize()
+        assert binding.tm_launch_count() == launches + (3 if any(sp.out_bytes) else 0)
+        if any(sp.out_bytes):
+            assert sp.status() == 0
+        for p, ((whole, _), f, e) in enumerate(zip(bufs, flats, expect)):
+            assert np.array_equal(f.cpu().numpy(), e)
+            assert bool((whole[:G.GUARD + 2 * p] == G.GUARD_BYTE).all())
+            assert bool((whole[G.GUARD + 2 * p + e.size:] == G.GUARD_BYTE).all())
+        # insert: new data into [lo, hi) of every plane, everything else untouched
+        gen = torch.Generator("cuda").manual_seed(r + 7)
+        data = [torch.randint(0, 256, (e.size,), dtype=torch.uint8, device="cuda", generator=gen) for e in expect]
+        before = st.arena.clone() if st.arena is not None else None
+        sp.rebind(data)
+        sp.insert()
+        torch.cuda.synchronize()
+        for idx, h, d in zip(planes, host, data):
+            hh = [x.copy() for x in h]
+            oracle_mod.shard_insert(hh, [x.size for x in hh], st.specs[idx[0]].elem_size, r, D, d.cpu().numpy())
+            for i, x in zip(idx, hh):
+                assert np.array_equal(st.host_bytes(i), x)
+        if before is not None:
+            mask = torch.ones_like(before, dtype=torch.bool)
+            for idx in planes:
+                for i in idx:
+                    o = st.tensors[i].data_ptr() - st.arena.data_ptr()
+                    mask[o:o + st.specs[i].nbytes] = False
+            assert torch.equal(st.arena[mask], before[mask])
+    dup = [st0.descs_of(st0.plane_indices(layouts.PLANE_M))[:2] * 2]          # the same tensors twice: insert refused
+    sp = ShardPlanMover(dup, 0, 1)
+    launches = binding.tm_launch_count()
+    with pytest.raises(binding.TmError) as e:
+        sp.insert()
+    assert e.value.status == binding.TM_ERR_OVERLAP and binding.tm_launch_count() == launches
+
+
+def test_buckets_in_pinned_host_memory(oracle_mod):
+    """Host-memory tier: the packed buffer is mapped pinned host memory, so pack writes the buckets
+    over PCIe itself and unpack + verify reads them from there; tensors and checksums stay on the GPU."""
+    for state, B in ((layouts.materialize(layouts.role_config(0), "cuda"), 1 << 20),
+                     (layouts.materialize_adversarial(layouts.adversarial_specs(300, max_log2=16), "cuda", seed=3), 1 << 18)):
+        host = G.host_tensors(state)
+        exp_stream, exp_cks = oracle_mod.pack(host, B)
+        m = RoleMover(state.descs(), B)
+        pinned = torch.full((m.total_bytes + 2 * G.GUARD,), G.GUARD_BYTE, dtype=torch.uint8).pin_memory()
+        assert pinned.data_ptr() % 256 == 0
+        hb = pinned[G.GUARD:G.GUARD + m.total_bytes]
+        cks = m.alloc_checksums()
+        m.pack(hb, cks)
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        assert np.array_equal(hb.numpy(), exp_stream) and np.array_equal(G.u64(cks), exp_cks)
+        assert bool((pinned[:G.GUARD] == G.GUARD_BYTE).all()) and bool((pinned[G.GUARD + m.total_bytes:] == G.GUARD_BYTE).all())
+        target = layouts.blank_like(state)
+        um = RoleMover(target.descs(), B)
+        got = um.alloc_checksums()
+        um.unpack_verify(hb, got)
+        torch.cuda.synchronize()
+        assert um.status() == 0 and np.array_equal(G.u64(got), exp_cks)
+        for k in range(len(host)):
+            assert np.array_equal(target.host_bytes(k), host[k])
+
+
+def test_ring_kernel_waits_made_to_expire_leave_everything_in_bounds(oracle_mod):
+    """With the wait limit at its minimum (1 ns) the ring kernels' own producer, store and consumer
+    waits run out in the middle of real work.  Either outcome is fine — finished, or TM_ERR_TIMEOUT
+    reported through the status word — but nothing may be written out of bounds, the call must
+    return, and the very next normal launch must be exact."""
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    exp_stream, exp_cks = oracle_mod.pack(G.host_tensors(state), cfg.bucket_bytes)
+    try:
+        binding.tm_options_set(wait_limit_ns=1)
+        hasty = RoleMover(state.descs(), cfg.bucket_bytes)
+    finally:
+        binding.tm_options_set()
+    whole, buckets = G.guarded(hasty.total_bytes)
+    cks = hasty.alloc_checksums()
+    seen = set()
+    for _ in range(5):
+        hasty.pack(buckets, cks)
+        seen.add(hasty.status())
+        assert G.guards_intact(whole, hasty.total_bytes)
+    assert seen <= {0, binding.TM_ERR_TIMEOUT}
+    if seen == {0}:                                           # every wait happened to succeed at once
+        assert np.array_equal(buckets.cpu().numpy(), exp_stream)
+    normal = RoleMover(state.descs(), cfg.bucket_bytes)
+    normal.pack(buckets, cks)
+    torch.cuda.synchronize()
+    assert normal.status() == 0 and G.guards_intact(whole, normal.total_bytes)
+    assert np.array_equal(buckets.cpu().numpy(), exp_stream) and np.array_equal(G.u64(cks), exp_cks)

@@ -181,10 +181,10 @@ def test_wave_by_wave_pack_equals_single_plan_and_oracle(oracle_mod, wave_bytes)
     exp_stream, exp_cks = oracle_mod.pack(G.host_tensors(state), cfg.bucket_bytes)
     wm = WaveMover(state.descs(), cfg.bucket_bytes, wave_bytes)
     assert (wm.total_bytes, wm.n_buckets) == (exp_stream.size, exp_cks.size)
-    assert len(wm.waves) == -(-wm.n_buckets // max(1, wave_bytes // cfg.bucket_bytes))
+    assert wm.n_waves == -(-wm.n_buckets // max(1, wave_bytes // cfg.bucket_bytes))
     whole, buckets = G.guarded(wm.total_bytes)
     cks = torch.zeros(wm.n_buckets, dtype=torch.int64, device="cuda")
-    for i in reversed(range(len(wm.waves))):          # order does not matter: waves are independent
+    for i in reversed(range(wm.n_waves)):             # order does not matter: waves are independent
         wm.pack_wave(i, buckets, cks)
     torch.cuda.synchronize()
     assert G.guards_intact(whole, wm.total_bytes)
@@ -323,12 +323,13 @@ def test_bounded_staging_ring_reproduces_the_stream(oracle_mod):
     slots = [G.guarded(2 << 20) for _ in range(2)]
     cks = torch.zeros(wm.n_buckets, dtype=torch.int64, device="cuda")
     received = torch.empty(wm.total_bytes, dtype=torch.uint8, device="cuda")
-    for i, w in enumerate(wm.waves):
+    for i in range(wm.n_waves):
         whole, slot = slots[i % 2]
         slot.fill_(0x77)                                   # stale contents of the recycled slot
         n = wm.pack_wave_into(i, slot, cks)
         assert n == wm.wave_bytes(i) <= slot.numel()
-        received[w.stream_begin:w.stream_end].copy_(slot[:n])
+        begin, end = wm.wave_span(i)
+        received[begin:end].copy_(slot[:n])
         torch.cuda.synchronize()
         assert G.guards_intact(whole, 2 << 20)
         assert bool((slot[n:] == 0x77).all())              # nothing written past the wave

@@ -187,3 +187,175 @@ def test_work_list_tiles_the_stream_exactly(lib, oracle_mod, seed):
     assert pos == T and k == n
     for a, b_ in zip(items[:-1], items[1:]):                        # an item never mixes buckets
         assert len(set(pieces["bucket"][a:b_].tolist())) == 1
+
+
+def _random_role(rng, n_max=40, log_max=20):
+    n = int(rng.integers(1, n_max))
+    sizes = [8 * max(1, int(2 ** x) // 8) for x in rng.uniform(3, log_max, n)]
+    addr, descs = FAKE, []
+    for nb in sizes:
+        addr += 2 * int(rng.integers(0, 64))
+        descs.append((addr, nb, 4, 1))
+        addr += nb
+    return sizes, descs
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_range_plans_concatenate_to_the_whole_plan(lib, oracle_mod, seed):
+    """A role cut into runs of whole buckets: every range plan tiles its own slot exactly, and shifted
+    by its stream offset the ranges reproduce the oracle's layout of the complete stream."""
+    rng = np.random.default_rng(500 + seed)
+    sizes, descs = _random_role(rng)
+    B = 256 * int(rng.choice([1, 3, 16, 4096, 32768]))
+    off, T, nbuckets = oracle_mod.layout(sizes, B)
+    per = int(rng.integers(1, max(2, nbuckets // 2 + 1)))
+    covered = np.zeros(T, dtype=np.int8)                       # 1 data, 2 padding
+    src = np.full(T, -1, dtype=np.int64)                       # tensor address of every data byte
+    first, n_ranges = 0, 0
+    while first < nbuckets:
+        plan = binding.Plan(descs, B, first, per)
+        lo, hi = first * B, min((first + per) * B, T)
+        assert (plan.first_bucket, plan.stream_begin, plan.whole_bytes, plan.whole_buckets) == (first, lo, T, nbuckets)
+        assert (plan.total_bytes, plan.n_buckets) == (hi - lo, min(per, nbuckets - first))
+        assert plan.offsets() == [int(x) for x in off]
+        pieces, items = plan.pieces()
+        pos = 0
+        for p in pieces:
+            o, n, pad = int(p["off"]), int(p["nbytes"]), int(p["pad"])
+            assert o == pos                                     # data and padding tile the slot without a gap
+            b = o // B
+            assert int(p["bucket"]) == b and int(p["word0"]) == (o - b * B) // 8 and o + n + pad <= (b + 1) * B
+            assert not covered[lo + o:lo + o + n + pad].any()
+            covered[lo + o:lo + o + n] = 1
+            covered[lo + o + n:lo + o + n + pad] = 2
+            src[lo + o:lo + o + n] = int(p["tensor"]) + np.arange(n)
+            pos = o + n + pad
+        assert pos == hi - lo
+        for a, b_ in zip(items[:-1], items[1:]):
+            assert len(set(pieces["bucket"][a:b_].tolist())) == 1
+        first += per
+        n_ranges += 1
+    assert n_ranges == -(-nbuckets // per)
+    for k, n in enumerate(sizes):                             # data bytes sit where the oracle's layout puts them
+        o = int(off[k])
+        assert (covered[o:o + n] == 1).all() and np.array_equal(src[o:o + n], descs[k][0] + np.arange(n))
+        assert (covered[o + n:(o + n + 255) // 256 * 256] == 2).all()
+    assert int((covered == 1).sum()) == sum(sizes) and (covered != 0).all()
+    with pytest.raises(binding.TmError) as e:
+        binding.Plan(descs, B, nbuckets, 1)
+    assert e.value.status == binding.TM_ERR_ARG
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_emit_records_tile_the_shards_exactly(lib, oracle_mod, seed):
+    """The second destinations attached to the pack pieces: over all pieces (of one plan, or of the
+    range plans of a role) they write every byte of every shard output exactly once, from the tensor
+    byte the oracle's bounds name."""
+    rng = np.random.default_rng(900 + seed)
+    sizes, descs = _random_role(rng, n_max=30, log_max=19)
+    n = len(sizes)
+    cut = sorted(set(int(x) for x in rng.integers(0, n + 1, 3)) | {0, n})
+    planes = [(a, b - a) for a, b in zip(cut[:-1], cut[1:]) if b > a][:3]
+    D = int(rng.integers(1, 9))
+    r = int(rng.integers(0, D))
+    B = 256 * int(rng.choice([2, 64, 4096]))
+    _, T, nbuckets = oracle_mod.layout(sizes, B)
+    per = nbuckets if seed % 2 == 0 else max(1, nbuckets // 3)
+    outs_base = [FAKE + (1 << 40) + (p << 36) + 2 * p for p in range(len(planes))]
+    bounds = [oracle_mod.shard_bounds(sum(sizes[f:f + c]) // 4, r, D) for f, c in planes]
+    written = [np.zeros((hi - lo) * 4, dtype=np.int64) - 1 for lo, hi in bounds]
+    first = 0
+    while first < nbuckets:
+        plan = binding.Plan(descs, B, first, per)
+        elems, need = binding.tm_plan_attach_shards(plan, planes, r, D, outs_base, [1 << 36] * len(planes), None, 0, 0)
+        assert elems == [hi - lo for lo, hi in bounds] and need >= plan.workspace_bytes
+        pieces, _ = plan.pieces()
+        emits = plan.emits()
+        assert emits.size == pieces.size
+        for p, em in zip(pieces, emits):
+            if em["len"] == 0:
+                continue
+            assert int(em["begin"]) + int(em["len"]) <= int(p["nbytes"]) and em["len"] % 4 == 0
+            q = max(i for i, ob in enumerate(outs_base) if ob <= int(em["out"]))
+            o = int(em["out"]) - outs_base[q]
+            assert (written[q][o:o + int(em["len"])] == -1).all()
+            written[q][o:o + int(em["len"])] = int(p["tensor"]) + int(em["begin"]) + np.arange(int(em["len"]))
+        with pytest.raises(binding.TmError) as e:             # records computed, nothing uploaded
+            binding.tm_state_pack_emit(plan, FAKE + (1 << 50), 1 << 40, None, 0)
+        assert e.value.status == binding.TM_ERR_STATE
+        first += per
+    for (f, c), (lo, hi), w in zip(planes, bounds, written):
+        flat = np.concatenate([descs[k][0] + np.arange(sizes[k]) for k in range(f, f + c)])
+        assert np.array_equal(w, flat[lo * 4:hi * 4])
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_shard_plan_pieces_tile_the_outputs_exactly(lib, oracle_mod, seed):
+    """Work list of a bound shard plan: the pieces write [0, (hi-lo)*e) of every flat buffer exactly
+    once, from the tensor bytes the oracle's bounds name, never exceed the chunk size, and stay
+    inside their tensor."""
+    rng = np.random.default_rng(1300 + seed)
+    planes, D = [], int(rng.integers(1, 70))
+    r = int(rng.integers(0, D))
+    for e in (4, 2, 8)[:int(rng.integers(1, 4))]:
+        sizes, descs = _random_role(rng, n_max=25, log_max=19)
+        planes.append([(a + (e << 44), nb, e, 0) for a, nb, _, _ in descs])
+    sp = binding.ShardPlan(planes, r, D)
+    flats = [FAKE + (1 << 50) + (p << 40) + 2 * int(rng.integers(0, 8)) for p in range(len(planes))]
+    bounds = [oracle_mod.shard_bounds(sum(d[1] for d in pl) // pl[0][2], r, D) for pl in planes]
+    assert sp.elems == [hi - lo for lo, hi in bounds]
+    sp.bind(flats, [1 << 40] * len(planes), None, 0, 0)
+    pieces, items, base = sp.pieces()
+    chunk = binding.tm_options_get()["shard_chunk_bytes"]
+    assert base == min(f for f, (lo, hi) in zip(flats, bounds) if hi > lo) if any(hi > lo for lo, hi in bounds) else True
+    written = [np.zeros((hi - lo) * pl[0][2], dtype=np.int64) - 1 for (lo, hi), pl in zip(bounds, planes)]
+    for p in pieces:
+        addr, n = base + int(p["off"]), int(p["nbytes"])
+        assert 0 < n <= chunk and p["pad"] == 0
+        q = max(i for i, f in enumerate(flats) if f <= addr)
+        o = addr - flats[q]
+        assert (written[q][o:o + n] == -1).all()
+        written[q][o:o + n] = int(p["tensor"]) + np.arange(n)
+        assert any(d[0] <= int(p["tensor"]) and int(p["tensor"]) + n <= d[0] + d[1] for d in planes[q])
+    for pl, (lo, hi), w in zip(planes, bounds, written):
+        e = pl[0][2]
+        flat = np.concatenate([d[0] + np.arange(d[1]) for d in pl])
+        assert np.array_equal(w, flat[lo * e:hi * e])
+    assert items[0] == 0 and items[-1] == pieces.size
+    if pieces.size:
+        with pytest.raises(binding.TmError) as ex:              # list built on the host only: nothing to launch with
+            sp.extract(0)
+        assert ex.value.status == binding.TM_ERR_STATE
+    else:
+        sp.extract(0)                                           # every shard empty: nothing to do
+
+
+def test_options_round_trip_and_validation(lib):
+    d = binding.tm_options_get()
+    assert d["chunk_bytes"] == 256 * 1024 and d["shard_chunk_bytes"] == 64 * 1024 and d["wait_limit_ns"] == 2_000_000_000
+    try:
+        binding.tm_options_set(chunk_bytes=8192, small_bytes=1024)
+        assert binding.tm_options_get()["chunk_bytes"] == 8192
+        plan = binding.Plan(_descs([40000]), 1 << 20)
+        pieces, _ = plan.pieces()
+        assert pieces["nbytes"].tolist() == [8192, 8192, 8192, 8192, 40000 - 4 * 8192]
+        for bad, code in ((dict(chunk_bytes=1000), binding.TM_ERR_ARG), (dict(chunk_bytes=4096 + 2), binding.TM_ERR_ALIGN),
+                          (dict(wait_limit_ns=0), binding.TM_ERR_ARG), (dict(ring_ctas_per_sm=3), binding.TM_ERR_ARG),
+                          (dict(group_max=0), binding.TM_ERR_ARG)):
+            with pytest.raises(binding.TmError) as e:
+                binding.tm_options_set(**bad)
+            assert e.value.status == code
+        assert binding.tm_options_get()["chunk_bytes"] == 8192     # a refused set changes nothing
+    finally:
+        binding.tm_options_set()
+    assert binding.tm_options_get() == d
+
+
+def test_plan_refuses_sizes_whose_sum_could_wrap(lib):
+    big = [(FAKE, 1 << 46, 2, 0)] * 1025                          # 2^56 + 2^46 bytes of stream
+    with pytest.raises(binding.TmError) as e:
+        binding.Plan(big, 1 << 30)
+    assert e.value.status == binding.TM_ERR_ARG
+    with pytest.raises(binding.TmError) as e:
+        binding.tm_shard_workspace(big, 0, 2)
+    assert e.value.status == binding.TM_ERR_ARG

@@ -18,6 +18,11 @@ pytestmark = pytest.mark.gpu
 GUARD = 512
 
 
+def _oracle_shard(oracle, state, indices, r, D):
+    host = [state.host_bytes(i) for i in indices]
+    return oracle.shard(host, [h.size for h in host], state.specs[indices[0]].elem_size, r, D)
+
+
 def _both_ways(descs, r, D, misalign=0):
     """(bytes from tm_shard_extract, bytes from tm_shard_extract_static, guard bands intact)."""
     stream = torch.cuda.current_stream().cuda_stream
@@ -33,7 +38,7 @@ def _both_ways(descs, r, D, misalign=0):
     return ref.cpu().numpy(), out.cpu().numpy(), intact
 
 
-def test_static_scratch_shard_matches_workspace_shard_twice_in_a_row():
+def test_static_scratch_shard_matches_workspace_shard_twice_in_a_row(oracle_mod):
     assert torch.cuda.is_available()
     binding.load_library()
     torch.cuda.set_device(0)
@@ -41,10 +46,14 @@ def test_static_scratch_shard_matches_workspace_shard_twice_in_a_row():
     # first call: a long list (config 0's fp32 master plane, mid-tensor shard boundaries)
     cfg = layouts.role_config(0)
     state = layouts.materialize(cfg, "cuda")
-    plane = [state.descs()[i] for i in state.plane_indices(layouts.PLANE_MASTER)]
+    master = state.plane_indices(layouts.PLANE_MASTER)
+    plane = [state.descs()[i] for i in master]
     ref, got, intact = _both_ways(plane, 1, 3)
     assert ref.size == 4 * (2 * 1_842_176 // 3 - 1_842_176 // 3) and intact
     assert np.array_equal(ref, got)
+    # and against the CPU oracle directly: the two entry points share the host planner, so agreeing
+    # with each other would not show a mistake made there
+    assert np.array_equal(got, _oracle_shard(oracle_mod, state, master, 1, 3))
     # second call, straight after: a shorter list of awkward pieces at 2-byte-granular addresses, so
     # most of the first call's list is still sitting in the array behind it
     odd = layouts.materialize_adversarial(layouts.odd_specs(7, n_tensors=12), "cuda", seed=7)
@@ -53,9 +62,11 @@ def test_static_scratch_shard_matches_workspace_shard_twice_in_a_row():
         if idx:
             ref, got, intact = _both_ways([odd.descs()[i] for i in idx], 2, 5, misalign=6)
             assert intact and np.array_equal(ref, got)
+            assert np.array_equal(got, _oracle_shard(oracle_mod, odd, idx, 2, 5))
     # and the first request again
     ref, got, intact = _both_ways(plane, 1, 3)
     assert intact and np.array_equal(ref, got)
+    assert np.array_equal(got, _oracle_shard(oracle_mod, state, master, 1, 3))
     assert binding.tm_launch_count() > launches
 
 
