@@ -348,6 +348,109 @@ int tm_checksum(const void* d_bytes, uint64_t nbytes, uint64_t bucket_bytes,
  * tm_workspace_status(d_workspace) yields TM_ERR_TIMEOUT.  d_workspace: >= 256 bytes, 256-byte aligned. */
 int tm_selftest_bounded_wait(void* d_workspace, uint64_t limit_ns, void* stream);
 
+/* ---- leaver -> joiner transfer through a bounded ring of staging slots ------------------------- */
+
+/* §7 "State Synchronization" delivers a role's state one-to-one from a leaver to its joiner, and
+ * §8.5 "Zero Memory Overhead Workflow" sends it through a per-pair channel that is created for the
+ * transfer and recycled, not through a second role-sized buffer.  Here the role is cut into waves of
+ * `buckets_per_wave` whole buckets (range plans); wave j of a round travels in slot j mod n_slots of a
+ * ring on each side.  Sender: pack wave -> slot (with the checksums of its buckets), hand slot and
+ * checksums to the transport, reuse the slot once the transport has read it.  Receiver: take a wave
+ * into a free slot, unpack + verify it (tm_state_unpack_verify), reuse the slot.  At the end of a
+ * round the receiver compares the checksums it recomputed with the sender's, bucket by bucket, and
+ * reports the waves that hold a mismatch; the sender packs and sends those again (the leaver's
+ * tensors are still there), up to max_rounds rounds in all.  Packing, sending, receiving and
+ * unpacking of different waves overlap: each side runs on two streams and only the slot hand-overs
+ * are ordered (events).  The integrity check and the re-request are this library's; the paper has
+ * none. */
+
+/* How bytes and control messages travel between the two sides.  All functions return 0 on success;
+ * anything else ends the transfer with that value if it is a negative tm_status, else with
+ * TM_ERR_TRANSPORT.  send / recv enqueue on `stream` (they may block the host until the peer has posted
+ * the matching call, as a rendezvous transport does) and move `nbytes` bytes of a slot plus
+ * `n_checksums` uint64 values; the data must land in the receiver's own memory.  Reports are small
+ * host-side messages: the list of waves to send again (n == 0: the round was clean). */
+typedef struct tm_transport {
+  void* ctx;
+  int (*send)(void* ctx, uint32_t wave, const void* d_slot, uint64_t nbytes, const uint64_t* d_checksums,
+              uint64_t n_checksums, void* stream);
+  int (*recv)(void* ctx, uint32_t wave, void* d_slot, uint64_t nbytes, uint64_t* d_checksums, uint64_t n_checksums,
+              void* stream);
+  int (*send_report)(void* ctx, const uint32_t* waves, uint32_t n);
+  int (*recv_report)(void* ctx, uint32_t* waves, uint32_t capacity, uint32_t* n);
+} tm_transport;
+
+typedef struct tm_xfer_stats {
+  uint32_t rounds;        /* rounds run (1 = nothing had to be sent again) */
+  uint32_t waves;         /* waves packed and sent / received and unpacked, all rounds */
+  uint32_t waves_again;   /* of those, in rounds after the first */
+  uint32_t bad_buckets;   /* receiver: buckets whose checksums differed, all rounds */
+  uint64_t first_bad_bucket;  /* receiver: the first of them (bucket index in the complete stream); ~0 if none */
+  uint64_t bytes;         /* slot bytes moved, all rounds */
+} tm_xfer_stats;
+
+/* The protocol itself, free of CUDA: the order of steps, the slot assignment (wave j of a round uses
+ * slot j mod n_slots), the rounds and the re-request.  tm_xfer_send / tm_xfer_receive run it with
+ * the library's kernels and a tm_transport; a harness can run the same loops over any other
+ * implementation of the steps (the CPU tests drive two processes over a host transport this way).
+ * Every hook returns 0 on success.  Sender hooks: pack, send, recv_report.  Receiver hooks: recv,
+ * unpack_verify, bad_waves (waits for the round's work, then lists which of `waves` arrived damaged),
+ * send_report.  Unused hooks may be NULL. */
+typedef struct tm_xfer_hooks {
+  void* ctx;
+  int (*pack)(void* ctx, uint32_t wave, uint32_t slot);
+  int (*send)(void* ctx, uint32_t wave, uint32_t slot);
+  int (*recv_report)(void* ctx, uint32_t* waves, uint32_t capacity, uint32_t* n);
+  int (*recv)(void* ctx, uint32_t wave, uint32_t slot);
+  int (*unpack_verify)(void* ctx, uint32_t wave, uint32_t slot);
+  int (*bad_waves)(void* ctx, const uint32_t* waves, uint32_t n_waves, uint32_t* bad, uint32_t* n_bad);
+  int (*send_report)(void* ctx, const uint32_t* waves, uint32_t n);
+} tm_xfer_hooks;
+
+/* Return TM_OK when a round ended clean, TM_ERR_VERIFY when waves were still damaged after
+ * max_rounds rounds, TM_ERR_TRANSPORT (or the hook's own negative status) when a hook failed or a
+ * report named a wave that was not sent in that round.  `stats` may be NULL. */
+int tm_xfer_run_sender(uint32_t n_waves, uint32_t n_slots, uint32_t max_rounds, const tm_xfer_hooks* hooks,
+                       tm_xfer_stats* stats);
+int tm_xfer_run_receiver(uint32_t n_waves, uint32_t n_slots, uint32_t max_rounds, const tm_xfer_hooks* hooks,
+                         tm_xfer_stats* stats);
+
+/* One side of a transfer: the role's tensors (sources on the sender, destinations on the receiver),
+ * cut into waves.  Host only; `descs` is copied. */
+typedef struct tm_xfer tm_xfer;
+int tm_xfer_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, uint64_t buckets_per_wave,
+                   uint32_t n_slots, tm_xfer** out);
+/* All outputs may be NULL: number of waves, bytes of one slot (buckets_per_wave * bucket_bytes), bytes
+ * of the ring (n_slots slots — the whole staging footprint of this side), device scratch for the
+ * waves' work lists, bucket count of the complete stream. */
+int tm_xfer_query(const tm_xfer* x, uint32_t* n_waves, uint64_t* slot_bytes, uint64_t* ring_bytes,
+                  uint64_t* workspace_bytes, uint64_t* n_buckets);
+/* Gives the side its memory (caller-owned, 256-byte aligned): the ring, the scratch (work lists are
+ * uploaded on `stream`), d_checksums (n_buckets uint64: filled by packing on the sender, recomputed
+ * from what arrived on the receiver) and, on the receiver, d_peer_checksums (n_buckets uint64: the
+ * sender's values as received; NULL on the sender).  Creates the events that order slot hand-overs. */
+int tm_xfer_bind(tm_xfer* x, void* d_ring, uint64_t ring_bytes, void* d_workspace, uint64_t workspace_bytes,
+                 uint64_t* d_checksums, uint64_t* d_peer_checksums, void* stream);
+/* Run one side to the end.  Packing (unpacking) is enqueued on the first stream, the transport's
+ * send (recv) on the second; the two must differ for the steps to overlap.  The calls block the host
+ * until the last round's report has been exchanged; the receiver's tensors are complete when
+ * tm_xfer_receive returns TM_OK. */
+int tm_xfer_send(tm_xfer* x, const tm_transport* transport, void* pack_stream, void* send_stream,
+                 uint32_t max_rounds, tm_xfer_stats* stats);
+int tm_xfer_receive(tm_xfer* x, const tm_transport* transport, void* unpack_stream, void* recv_stream,
+                    uint32_t max_rounds, tm_xfer_stats* stats);
+void tm_xfer_destroy(tm_xfer* x);
+
+/* Transport between two sides that live in one process on one GPU (two host threads): send waits for
+ * the matching recv to be posted, then copies slot and checksums device-to-device on its stream into
+ * the receiver's slot; reports go through a mailbox.  It stands in for a link between two GPUs, whose
+ * transport (for example NCCL send / recv of whole slots) implements the same four functions.  A
+ * posted call that finds no partner within 60 s fails with TM_ERR_TRANSPORT.  *transport is filled
+ * with functions and a context that stay valid until tm_loopback_destroy. */
+typedef struct tm_loopback tm_loopback;
+int tm_loopback_create(tm_loopback** out, tm_transport* transport);
+void tm_loopback_destroy(tm_loopback* lb);
+
 /* One piece of a plan's work list, as the kernels see it (for inspection and host-side checks). */
 typedef struct tm_piece {
   uint64_t tensor;   /* device address of the piece's first tensor byte */

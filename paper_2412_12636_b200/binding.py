@@ -37,6 +37,16 @@ SIGNATURES = {
     "tm_shard_plan_status": (_int, [_p, _p, _p]),
     "tm_shard_plan_pieces": (_int, [_p, _p, _u64, _p, _p, _u64, _p, _p]),
     "tm_shard_plan_destroy": (None, [_p]),
+    "tm_xfer_run_sender": (_int, [_u32, _u32, _u32, _p, _p]),
+    "tm_xfer_run_receiver": (_int, [_u32, _u32, _u32, _p, _p]),
+    "tm_xfer_create": (_int, [_p, _u64, _u64, _u64, _u32, _p]),
+    "tm_xfer_query": (_int, [_p, _p, _p, _p, _p, _p]),
+    "tm_xfer_bind": (_int, [_p, _p, _u64, _p, _u64, _p, _p, _p]),
+    "tm_xfer_send": (_int, [_p, _p, _p, _p, _u32, _p]),
+    "tm_xfer_receive": (_int, [_p, _p, _p, _p, _u32, _p]),
+    "tm_xfer_destroy": (None, [_p]),
+    "tm_loopback_create": (_int, [_p, _p]),
+    "tm_loopback_destroy": (None, [_p]),
     "tm_plan_offsets": (_int, [_p, _p]),
     "tm_plan_pieces": (_int, [_p, _p, _u64, _p, _p, _u64, _p]),
     "tm_plan_upload": (_int, [_p, _p, _u64, _p]),
@@ -70,6 +80,36 @@ class TmOptions(ctypes.Structure):
     _fields_ = [("chunk_bytes", _u64), ("shard_chunk_bytes", _u64), ("small_bytes", _u64), ("group_bytes", _u64),
                 ("cksum_tile_bytes", _u64), ("wait_limit_ns", _u64), ("group_max", _u32), ("ring_ctas_per_sm", _u32),
                 ("ctas_per_sm", _u32), ("reserved", _u32)]
+
+
+# callback types of tm_transport and tm_xfer_hooks
+SEND_FN = ctypes.CFUNCTYPE(_int, _p, _u32, _p, _u64, _p, _u64, _p)
+RECV_FN = ctypes.CFUNCTYPE(_int, _p, _u32, _p, _u64, _p, _u64, _p)
+SEND_REPORT_FN = ctypes.CFUNCTYPE(_int, _p, ctypes.POINTER(_u32), _u32)
+RECV_REPORT_FN = ctypes.CFUNCTYPE(_int, _p, ctypes.POINTER(_u32), _u32, ctypes.POINTER(_u32))
+STEP_FN = ctypes.CFUNCTYPE(_int, _p, _u32, _u32)
+BAD_WAVES_FN = ctypes.CFUNCTYPE(_int, _p, ctypes.POINTER(_u32), _u32, ctypes.POINTER(_u32), ctypes.POINTER(_u32))
+
+
+class TmTransport(ctypes.Structure):
+    _fields_ = [("ctx", _p), ("send", SEND_FN), ("recv", RECV_FN), ("send_report", SEND_REPORT_FN),
+                ("recv_report", RECV_REPORT_FN)]
+
+
+class TmXferHooks(ctypes.Structure):
+    _fields_ = [("ctx", _p), ("pack", STEP_FN), ("send", STEP_FN), ("recv_report", RECV_REPORT_FN), ("recv", STEP_FN),
+                ("unpack_verify", STEP_FN), ("bad_waves", BAD_WAVES_FN), ("send_report", SEND_REPORT_FN)]
+
+
+class TmXferStats(ctypes.Structure):
+    _fields_ = [("rounds", _u32), ("waves", _u32), ("waves_again", _u32), ("bad_buckets", _u32),
+                ("first_bad_bucket", _u64), ("bytes", _u64)]
+
+    def as_dict(self) -> dict:
+        d = {name: getattr(self, name) for name, _ in self._fields_}
+        if d["first_bad_bucket"] == (1 << 64) - 1:
+            d["first_bad_bucket"] = None
+        return d
 
 
 class TmError(RuntimeError):

@@ -123,6 +123,43 @@ def test_full_size_role_configs(oracle_mod, idx):
         assert out.numel() == 4 * expect_elems
 
 
+def test_config3_fused_send_and_ring_transfer_at_full_size(oracle_mod):
+    """Config 3 at full size, the two fused forms the benchmark times.  (1) pack + checksum + the three
+    shards in one launch: stream and checksums equal the plain pack's (itself checked against the
+    oracle above), sampled buckets and the complete shards are compared with the oracle.  (2) the
+    role travels through a ring of two 1 GiB slots per side (loopback transport): the receiver's
+    tensors equal the sender's and every checksum equals the plain pack's."""
+    from paper_2412_12636_b200 import transfer
+    cfg = layouts.role_config(3)
+    state = layouts.materialize(cfg, "cuda")
+    mover, buckets, cks = G.gpu_pack(state)
+    plain = buckets.clone()
+    buckets.zero_()
+    P = len(cfg.model)
+    planes = [(P, P), (2 * P, P), (3 * P, P)]
+    outs = mover.attach_shards(planes, cfg.shard_r, cfg.shard_D)
+    fused = mover.alloc_checksums()
+    mover.pack_emit(buckets, fused)
+    torch.cuda.synchronize()
+    assert mover.status() == 0
+    assert torch.equal(buckets, plain) and np.array_equal(G.u64(fused), cks)
+    del plain
+    nb = mover.n_buckets
+    check_sampled_buckets(oracle_mod, state, mover, buckets, G.u64(fused), sorted({0, nb // 3, nb - 1}))
+    for (first, count), out in zip(planes, outs):
+        idx = list(range(first, first + count))
+        ref = check_shard_sampled(oracle_mod, state, idx, cfg.shard_r, cfg.shard_D)   # oracle-checked extract
+        assert out.numel() == 4 * 44_571_307 and torch.equal(out, ref)
+    del buckets, outs, mover
+    torch.cuda.empty_cache()
+    target = layouts.blank_like(state)
+    tx, rx, ms = transfer.loopback_transfer(state.descs(), target.descs(), cfg.bucket_bytes, 4, 2)
+    assert tx.n_waves == 14 and tx.ring_bytes == 2 << 30 and rx.stats["rounds"] == 1 and rx.stats["bad_buckets"] == 0
+    assert np.array_equal(G.u64(tx.checksums), cks) and np.array_equal(G.u64(rx.checksums), cks)
+    for a, b in zip(state.tensors, target.tensors):
+        assert torch.equal(layouts.tensor_bytes(a), layouts.tensor_bytes(b))
+
+
 def test_config1_norm_vectors_are_ones_closed_form(oracle_mod):
     # config 1 sets RMSNorm weights to 1.0: a bucket holding only a 2048-element fp32 norm vector at
     # word s has checksum c*((s+1024)^2 - s^2), c = 0x3F8000003F800000; checked through the library

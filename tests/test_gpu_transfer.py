@@ -1,0 +1,106 @@
+"""Leaver -> joiner transfer on one GPU through the loopback transport: the role is packed wave by
+wave into a small ring of slots, copied into the receiver's ring, unpacked and verified there, with
+all four stages overlapping.  The receiver's tensors and both sides' checksums must equal the CPU
+oracle's; a wave damaged in flight must be detected, re-requested and repaired."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_12636_b200 import binding, layouts, transfer
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _cuda():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.load_library()
+    torch.cuda.set_device(0)
+    yield
+
+
+def _flip_on_host(hits, seen):
+    """after_recv hook: for every (round-trip count, wave) in `hits`, copy the arrived slot to the host,
+    flip one bit of the host copy, and copy it back — on the stream the slot arrived on."""
+    def hook(rx, wave, d_slot, nbytes, stream):
+        seen[wave] = seen.get(wave, 0) + 1
+        byte = hits.get((seen[wave], wave))
+        if byte is None:
+            return
+        off = d_slot - rx.ring.data_ptr()
+        view = rx.ring[off:off + nbytes]
+        with torch.cuda.stream(torch.cuda.ExternalStream(stream)):
+            host = view.cpu()
+            host[byte % nbytes] ^= 0x20
+            view.copy_(host)
+    return hook
+
+
+def _check_receiver(oracle, state, target, tx, rx, B):
+    host = G.host_tensors(state)
+    _, exp_cks = oracle.pack(host, B)
+    assert np.array_equal(G.u64(tx.checksums), exp_cks) and np.array_equal(G.u64(rx.checksums), exp_cks)
+    assert np.array_equal(G.u64(rx.peer_checksums), exp_cks)
+    if target.arena is not None:
+        exp_arena = np.full(target.arena.numel(), 0xA5, dtype=np.uint8)
+        for t, h in zip(target.tensors, host):
+            o = t.data_ptr() - target.arena.data_ptr()
+            exp_arena[o:o + h.size] = h
+        assert np.array_equal(target.arena.cpu().numpy(), exp_arena)
+    else:
+        for k, h in enumerate(host):
+            assert np.array_equal(target.host_bytes(k), h), f"tensor {k}"
+
+
+@pytest.mark.parametrize("per_wave,n_slots", [(1, 2), (3, 2), (4, 3), (64, 1)])
+def test_loopback_transfer_config0(oracle_mod, per_wave, n_slots):
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    target = layouts.blank_like(state)
+    tx, rx, ms = transfer.loopback_transfer(state.descs(), target.descs(), cfg.bucket_bytes, per_wave, n_slots)
+    n_waves = -(-25 // per_wave)
+    assert tx.n_waves == rx.n_waves == n_waves and tx.ring_bytes == n_slots * per_wave * cfg.bucket_bytes
+    for side in (tx, rx):
+        assert side.stats["rounds"] == 1 and side.stats["waves"] == n_waves and side.stats["bad_buckets"] == 0
+        assert side.stats["bytes"] == 25_790_464
+    _check_receiver(oracle_mod, state, target, tx, rx, cfg.bucket_bytes)
+
+
+def test_loopback_transfer_adversarial_layout(oracle_mod):
+    state = layouts.materialize_adversarial(layouts.adversarial_specs(800, max_log2=17), "cuda", seed=17)
+    target = layouts.blank_like(state)
+    tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), 1 << 18, 3, 2)
+    assert rx.stats["rounds"] == 1
+    _check_receiver(oracle_mod, state, target, tx, rx, 1 << 18)
+
+
+def test_wave_damaged_in_flight_is_detected_and_sent_again(oracle_mod):
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    target = layouts.blank_like(state)
+    seen = {}
+    # wave 2 arrives damaged in round 1 (bucket 7 of the stream), wave 5 in rounds 1 and 2
+    hits = {(1, 2): 1 * cfg.bucket_bytes + 12345, (1, 5): 77, (2, 5): 2 * cfg.bucket_bytes + 5}
+    tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), cfg.bucket_bytes, 3, 2, max_rounds=4,
+                                           after_recv=_flip_on_host(hits, seen))
+    for side in (tx, rx):
+        assert side.stats["rounds"] == 3 and side.stats["waves"] == 9 + 2 + 1 and side.stats["waves_again"] == 3
+    assert rx.stats["bad_buckets"] == 3 and rx.stats["first_bad_bucket"] == 7
+    assert seen[2] == 2 and seen[5] == 3 and seen[0] == 1
+    _check_receiver(oracle_mod, state, target, tx, rx, cfg.bucket_bytes)
+
+
+def test_transfer_reports_failure_when_damage_persists(oracle_mod):
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    target = layouts.blank_like(state)
+    hits = {(k, 1): 3 for k in range(1, 6)}
+    with pytest.raises(binding.TmError) as e:
+        transfer.loopback_transfer(state.descs(), target.descs(), cfg.bucket_bytes, 5, 2, max_rounds=2,
+                                   after_recv=_flip_on_host(hits, {}))
+    assert e.value.status == binding.TM_ERR_VERIFY and e.value.stats["rounds"] == 2
+    # the context is fine afterwards
+    tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), cfg.bucket_bytes, 5, 2)
+    _check_receiver(oracle_mod, state, target, tx, rx, cfg.bucket_bytes)
