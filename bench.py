@@ -294,7 +294,7 @@ def run_reference(args) -> None:
 class RoleBench:
     """One role on the current GPU with every buffer the step needs."""
 
-    def __init__(self, workload: str, prepared=None, layers: Optional[int] = None):
+    def __init__(self, workload: str, prepared=None, layers: Optional[int] = None, shard: Optional[Tuple[int, int]] = None):
         from paper_2412_12636_b200 import layouts
         from paper_2412_12636_b200.mover import MultiShardExtractor, RoleMover, ShardExtractor, ShardPlanMover
         if prepared is not None:      # (RoleState, bucket_bytes, r, D): a wave of a larger role
@@ -309,6 +309,8 @@ class RoleBench:
             cfg = layouts.role_config(WORKLOADS[workload], layers=layers)
             self.state = layouts.materialize(cfg, "cuda")
             self.name, self.bucket_bytes, self.shard_r, self.shard_D = cfg.name, cfg.bucket_bytes, cfg.shard_r, cfg.shard_D
+            if shard is not None:
+                self.shard_r, self.shard_D = shard
             planes = [self.state.plane_indices(p) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)]
         state = self.state
         self.target = layouts.blank_like(state)
@@ -592,7 +594,8 @@ def run_ours(args) -> None:
     if use_dist:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    role = RoleBench(args.workload, layers=args.layers)
+    shard = tuple(int(x) for x in args.shard.split(",")) if args.shard else None
+    role = RoleBench(args.workload, layers=args.layers, shard=shard)
     for _ in range(max(args.warmup, 3)):
         role.one_step()
     torch.cuda.synchronize()
@@ -631,7 +634,7 @@ def run_ours(args) -> None:
     cpu_baseline = None
     also = {}
     transfer_entry = host_tier = None
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.kernels_only:
         per_wave = max(1, (1 << 30) // role.bucket_bytes)          # 1 GiB slots (config 0: the whole role in one)
         transfer_entry = role.time_transfer(per_wave, 2)
         ok = ok and transfer_entry["outputs_match"]
@@ -649,7 +652,7 @@ def run_ours(args) -> None:
     state_bytes, n_buckets, n_tensors = role.state.state_bytes, role.mover.n_buckets, len(role.state.specs)
     name, bucket_bytes, shard = role.name, role.bucket_bytes, f"r={role.shard_r} of D={role.shard_D}"
     bytes_per_step = role.bytes_per_step
-    if rank == 0 and world == 1 and args.also:
+    if rank == 0 and world == 1 and args.also and not args.kernels_only:
         del role
         torch.cuda.empty_cache()
         for w in args.also.split(","):
@@ -852,7 +855,13 @@ def main() -> None:
     ap.add_argument("--layers", type=int, default=None,
                     help="reduce cfg0..cfg3 to their first LAYERS transformer layers: a small, self-ending case "
                          "(a few GB, still far larger than the L2) for profiler captures")
+    ap.add_argument("--shard", default="", help="R,D: override the workload's shard rank and count (cfg0..cfg3)")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="only the kernels of the step and of the fused calls: no transfer pipeline, host tier, "
+                         "end-to-end leg, CPU baseline or second workload (with --layers: the case profiler captures run)")
     args = ap.parse_args()
+    if args.kernels_only:
+        args.no_e2e = args.no_cpu_baseline = True
     if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         raise SystemExit(launch_local_ranks(args.gpus))
     if args.impl == "reference":

@@ -276,6 +276,60 @@ def test_adversarial_200000_tensors_in_waves(oracle_mod):
     assert sum(c.size for c in all_cks) == nb
 
 
+def test_config4_whole_fp32_plane_every_rank_of_64(oracle_mod):
+    """Config 4's shard requirement as written: the fp32 tensors of the complete 200 000-tensor set form
+    one plane (about 73 GB); shard r of 64 is extracted for every r and the 64 outputs are compared,
+    on the device, with the matching slices of the source tensors — exact union coverage of the whole
+    plane — and three ranks with the oracle.  Only the fp32 tensors are materialised, in chunks."""
+    from paper_2412_12636_b200.mover import ShardPlanMover
+    specs = [s for s in layouts.adversarial_specs(200_000) if s.elem_size == 4]
+    chunks, tensors, chunk, acc = [], [], [], 0
+    for s in specs:
+        chunk.append(s)
+        acc += s.nbytes
+        if acc > (8 << 30):
+            chunks.append(chunk)
+            chunk, acc = [], 0
+    if chunk:
+        chunks.append(chunk)
+    arenas = []
+    for ci, ch in enumerate(chunks):
+        part = layouts.materialize_adversarial(ch, "cuda", wave=1000 + ci)     # 2-byte-granular addresses
+        arenas.append(part.arena)
+        tensors.extend(part.tensors)
+        del part
+        torch.cuda.empty_cache()
+    state = layouts.RoleState("cfg4-fp32-plane", specs, tensors, layouts.ADVERSARIAL_BUCKET, 0, 64)
+    idx = list(range(len(specs)))
+    descs = state.descs()
+    counts = [s.numel for s in specs]
+    N = sum(counts)
+    starts = np.concatenate([[0], np.cumsum(counts)])
+    assert N * 4 > 60 << 30
+    cap = 4 * (N // 64 + 1)
+    whole, out = G.guarded(cap)
+    prev = 0
+    for r in range(64):
+        lo, hi = binding.tm_shard_bounds(N, r, 64)
+        assert (lo, hi) == oracle_mod.shard_bounds(N, r, 64) and lo == prev
+        prev = hi
+        sp = ShardPlanMover([descs], r, 64, flats=[out[:4 * (hi - lo)]])
+        sp.extract()
+        torch.cuda.synchronize()
+        assert sp.status() == 0 and G.guards_intact(whole, cap)
+        k0 = int(np.searchsorted(starts, lo, side="right")) - 1
+        k = k0
+        while k < len(specs) and starts[k] < hi:                      # slices of the tensors the shard crosses
+            a, b = max(lo, int(starts[k])), min(hi, int(starts[k + 1]))
+            src = tensors[k][4 * (a - int(starts[k])):4 * (b - int(starts[k]))]
+            assert torch.equal(out[4 * (a - lo):4 * (b - lo)], src), (r, k)
+            k += 1
+        del sp
+    assert prev == N
+    for r in (0, 29, 63):
+        check_shard_sampled(oracle_mod, state, idx, r, 64)
+
+
 def check_unpack_parts(state, buckets, B):
     """Unpack into fresh 0xA5-filled buffers, one per tensor part; returns them."""
     targets = [torch.full((t.numel(),), 0xA5, dtype=torch.uint8, device="cuda") for t in state.tensors]
