@@ -383,6 +383,24 @@ class RoleBench:
         return {"ms": round(ms, 4), "GB/s": round(gbs(nbytes, ms), 1),
                 "checksums_match": bool(torch.equal(got, self.cks_fused))}
 
+    def time_graph_step(self, steps: int) -> Dict[str, float]:
+        """The four launches of the step captured once in a CUDA graph and replayed: what the step costs
+        when the host's launch work is taken out (it matters for small roles)."""
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            self.one_step()
+        for _ in range(2):
+            g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(self.stream)
+        for _ in range(steps):
+            g.replay()
+        b.record(self.stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / steps
+        return {"ms_per_step": round(ms, 4), "GB/s": round(gbs(self.bytes_per_step, ms), 1), "outputs_match": self.self_check()}
+
     def time_shard_one_shot(self, steps: int) -> Dict[str, float]:
         """tm_shard_extract_planes (validates, builds and uploads its list on every call) against the
         reusable plan of the timed step."""
@@ -620,6 +638,8 @@ def run_ours(args) -> None:
     ok = ok and (fused_send is None or fused_send["outputs_match"])
     shard_one_shot = role.time_shard_one_shot(max(3, args.steps // 2)) if rank == 0 else None
     ok = ok and (shard_one_shot is None or shard_one_shot["outputs_match"])
+    graph_step = role.time_graph_step(args.steps) if rank == 0 else None
+    ok = ok and (graph_step is None or graph_step["outputs_match"])
 
     total_ms, total_bytes = aggregate_over_ranks(elapsed_ms, role.bytes_per_step * args.steps)
     peak, peak_kind = measured_hbm_peak()
@@ -635,7 +655,8 @@ def run_ours(args) -> None:
     also = {}
     transfer_entry = host_tier = None
     if rank == 0 and world == 1 and not args.kernels_only:
-        per_wave = max(1, (1 << 30) // role.bucket_bytes)          # 1 GiB slots (config 0: the whole role in one)
+        # slots of at most 1 GiB and at most an eighth of the role: two of them per side
+        per_wave = max(1, min((1 << 30) // role.bucket_bytes, role.mover.n_buckets // 8))
         transfer_entry = role.time_transfer(per_wave, 2)
         ok = ok and transfer_entry["outputs_match"]
         if not args.no_e2e:
@@ -692,6 +713,8 @@ def run_ours(args) -> None:
                                           separate_ms=round(ops["pack"]["ms"] + ops["shard"]["ms"], 4)),
         "shard_one_shot": shard_one_shot and dict(shard_one_shot, note="tm_shard_extract_planes: list built and uploaded on "
                                                   "every call; the timed step uses the reusable tm_shard_plan"),
+        "graph_step": graph_step and dict(graph_step, note="the step's four launches captured in one CUDA graph and replayed; "
+                                          "not the timed step"),
         "transfer": transfer_entry, "host_tier": host_tier,
         "also": also,
     }

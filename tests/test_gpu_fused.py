@@ -227,3 +227,49 @@ def test_ring_kernel_waits_made_to_expire_leave_everything_in_bounds(oracle_mod)
     torch.cuda.synchronize()
     assert normal.status() == 0 and G.guards_intact(whole, normal.total_bytes)
     assert np.array_equal(buckets.cpu().numpy(), exp_stream) and np.array_equal(G.u64(cks), exp_cks)
+
+
+def test_step_captured_in_a_cuda_graph_replays_exactly(oracle_mod):
+    """pack, checksum, unpack+verify and the plan-based shard extract enqueue only stream work once
+    their plans are uploaded, so the whole step can be captured in a CUDA graph.  The replayed graph
+    must give the oracle's results for whatever the source tensors hold at replay time."""
+    cfg = layouts.role_config(0)
+    state = layouts.materialize(cfg, "cuda")
+    target = layouts.blank_like(state)
+    mover, unmover = RoleMover(state.descs(), cfg.bucket_bytes), RoleMover(target.descs(), cfg.bucket_bytes)
+    whole, buckets = G.guarded(mover.total_bytes)
+    fused, alone, received = mover.alloc_checksums(), mover.alloc_checksums(), mover.alloc_checksums()
+    planes = [target.descs_of(target.plane_indices(p)) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)]
+    sp = ShardPlanMover(planes, cfg.shard_r, cfg.shard_D)
+
+    def step():
+        mover.pack(buckets, fused)
+        mover.checksum(buckets, alone)
+        unmover.unpack_verify(buckets, received)
+        sp.extract()
+
+    step()                                   # first launches outside the capture (one-time kernel attributes)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for trial in range(2):
+        for t in state.tensors:              # new contents: the graph must read the tensors, not a snapshot
+            layouts.tensor_bytes(t).random_(0, 256, generator=torch.Generator("cuda").manual_seed(trial * 7919 + t.numel()))
+        buckets.fill_(0xEE)
+        launches = binding.tm_launch_count()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert binding.tm_launch_count() == launches          # replayed by the driver, not launched by the library
+        host = G.host_tensors(state)
+        exp_stream, exp_cks = oracle_mod.pack(host, cfg.bucket_bytes)
+        assert np.array_equal(buckets.cpu().numpy(), exp_stream) and G.guards_intact(whole, mover.total_bytes)
+        for c in (fused, alone, received):
+            assert np.array_equal(G.u64(c), exp_cks)
+        for k in range(len(host)):
+            assert np.array_equal(target.host_bytes(k), host[k])
+        idxs = [state.plane_indices(p) for p in (layouts.PLANE_MASTER, layouts.PLANE_M, layouts.PLANE_V)]
+        for idx, out in zip(idxs, sp.flats):
+            sub = [host[i] for i in idx]
+            assert np.array_equal(out.cpu().numpy(), oracle_mod.shard(sub, [h.size for h in sub], 4, cfg.shard_r, cfg.shard_D))
+    assert mover.status() == 0 and unmover.status() == 0 and sp.status() == 0

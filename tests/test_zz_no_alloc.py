@@ -70,6 +70,45 @@ def test_static_scratch_shard_matches_workspace_shard_twice_in_a_row(oracle_mod)
     assert binding.tm_launch_count() > launches
 
 
+def test_static_scratch_calls_from_two_threads_on_one_stream(oracle_mod):
+    """The entry point documents that host threads sharing ONE stream may call it concurrently: the
+    clear / copy / copy / launch sequence of a call runs under one lock, so every kernel reads the
+    list its own call wrote.  Two threads issue different requests on the same stream many times."""
+    import threading
+    binding.load_library()
+    torch.cuda.set_device(0)
+    state = layouts.materialize(layouts.role_config(0), "cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    jobs = []
+    for plane, r, D in ((layouts.PLANE_MASTER, 1, 3), (layouts.PLANE_V, 4, 5)):
+        idx = state.plane_indices(plane)
+        expect = _oracle_shard(oracle_mod, state, idx, r, D)
+        descs = binding.make_descs([state.descs()[i] for i in idx])
+        outs = [torch.zeros(expect.size, dtype=torch.uint8, device="cuda") for _ in range(20)]
+        jobs.append((descs, r, D, outs, expect))
+    errors = []
+
+    def work(job):
+        descs, r, D, outs, expect = job
+        try:
+            torch.cuda.set_device(0)
+            for out in outs:
+                binding.tm_shard_extract_static(descs, r, D, out.data_ptr(), out.numel(), stream)
+        except Exception as e:
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for descs, r, D, outs, expect in jobs:
+        for out in outs:
+            assert np.array_equal(out.cpu().numpy(), expect)
+
+
 def test_static_scratch_refuses_what_does_not_fit():
     binding.load_library()
     stream = torch.cuda.current_stream().cuda_stream
