@@ -233,6 +233,14 @@ int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const
 int tm_state_pack_emit(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint64_t* d_checksums,
                        void* stream);
 
+/* The receiving side's counterpart (a joiner that is sent a whole role and keeps, under the distributed
+ * optimizer, its own slice of the optimizer state as flat buffers — §7 "State Synchronization"): does
+ * what tm_state_unpack_verify does (same arguments, same results, d_checksums required) and, from the
+ * same staged copy of every piece, also fills the shard outputs attached with tm_plan_attach_shards —
+ * one read of the received buckets gives the tensors, the checksums and the shards. */
+int tm_state_unpack_emit(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, uint64_t* d_checksums,
+                         void* stream);
+
 /* Host helper: floor shard bounds lo = floor(r*N/D), hi = floor((r+1)*N/D) in 128-bit arithmetic. */
 int tm_shard_bounds(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
 

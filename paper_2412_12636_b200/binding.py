@@ -57,6 +57,7 @@ SIGNATURES = {
     "tm_state_unpack_verify": (_int, [_p, _p, _u64, _p, _p]),
     "tm_plan_attach_shards": (_int, [_p, _p, _p, _u32, _u32, _u32, _p, _p, _p, _p, _u64, _p, _p]),
     "tm_state_pack_emit": (_int, [_p, _p, _u64, _p, _p]),
+    "tm_state_unpack_emit": (_int, [_p, _p, _u64, _p, _p]),
     "tm_shard_bounds": (_int, [_u64, _u32, _u32, _p, _p]),
     "tm_shard_workspace": (_int, [_p, _u64, _u32, _u32, _p]),
     "tm_shard_extract": (_int, [_p, _u64, _u32, _u32, _p, _u64, _p, _p, _u64, _p]),
@@ -283,6 +284,11 @@ def tm_plan_attach_shards(plan: Plan, planes: Sequence[Tuple[int, int]], r: int,
 def tm_state_pack_emit(plan: Plan, d_buckets: int, capacity: int, d_checksums: Optional[int], stream: int) -> None:
     _check(load_library().tm_state_pack_emit(plan.handle, d_buckets, capacity, d_checksums, stream),
            "tm_state_pack_emit")
+
+
+def tm_state_unpack_emit(plan: Plan, d_buckets: int, nbytes: int, d_checksums: int, stream: int) -> None:
+    _check(load_library().tm_state_unpack_emit(plan.handle, d_buckets, nbytes, d_checksums, stream),
+           "tm_state_unpack_emit")
 
 
 def tm_shard_bounds(n_elems: int, r: int, D: int) -> Tuple[int, int]:

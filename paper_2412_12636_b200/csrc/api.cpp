@@ -457,6 +457,24 @@ int tm_state_pack_emit(const tm_plan* plan, void* d_buckets, uint64_t capacity, 
   return e == 0 ? TM_OK : tms::cuda_fail(e);
 }
 
+int tm_state_unpack_emit(const tm_plan* plan, const void* d_buckets, uint64_t nbytes, uint64_t* d_checksums,
+                         void* stream) {
+  return guarded([&]() -> int {
+    if (d_checksums == nullptr) return TM_ERR_ARG;
+    int rc = check_buckets(plan, d_buckets, nbytes, d_checksums);
+    if (rc != TM_OK) return rc;
+    if (plan->d_emit_workspace == nullptr) return TM_ERR_STATE;
+    if ((rc = targets_ok(plan)) != TM_OK) return rc;
+    for (const auto& o : plan->emit_outs)
+      if (tms::ranges_overlap(o.first, o.second, (uint64_t)(uintptr_t)d_buckets, plan->total_bytes)) return TM_ERR_OVERLAP;
+    TM_CUDA(cudaMemsetAsync(d_checksums, 0, plan->n_buckets * sizeof(uint64_t), (cudaStream_t)stream));
+    tms::RingLaunch a = ring_args(plan, plan->d_emit_workspace, plan->emit_layout, const_cast<void*>(d_buckets), d_checksums);
+    a.d_emits = (const tms::Emit*)(plan->d_emit_workspace + plan->emit_layout.emits_off);
+    int e = tms::launch_ring(tms::kRingToTensorsVerifyEmit, a, stream);
+    return e == 0 ? TM_OK : tms::cuda_fail(e);
+  });
+}
+
 int tm_selftest_bounded_wait(void* d_workspace, uint64_t limit_ns, void* stream) {
   if (d_workspace == nullptr || limit_ns == 0 || limit_ns > 5000000000ull) return TM_ERR_ARG;
   if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;

@@ -193,9 +193,9 @@ __device__ __forceinline__ void emit_direct(const Emit& em, const uint8_t* piece
 // given by TO_TENSORS (PACK implies TO_TENSORS == false).  VERIFY (with TO_TENSORS): the unpack also
 // accumulates the per-bucket checksums of the stream it reads — data and padding bytes as they
 // arrived — so that a receiver checks and scatters in one pass over the buckets.
-// EMIT (with PACK): emits[i] gives piece i an optional second destination for a sub-range of its
-// bytes; the consumers write it from the stage in shared memory (bulk pieces) or re-read the few KiB
-// of a small piece they have just copied (served by L1 / L2).
+// EMIT (with PACK, or with TO_TENSORS + VERIFY): emits[i] gives piece i an optional second destination
+// for a sub-range of its bytes; the consumers write it from the stage in shared memory (bulk pieces)
+// or re-read the few KiB of a small piece they have just copied (served by L1 / L2).
 template <bool PACK, bool TO_TENSORS, bool VERIFY, bool EMIT>
 __global__ void __launch_bounds__(kRingThreads, 1)
 ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_first, uint32_t n_items,
@@ -348,6 +348,11 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
           uint8_t* t = reinterpret_cast<uint8_t*>(s.tensor);
           uint8_t* f = flat + s.off;
           copy_piece(TO_TENSORS ? t : f, TO_TENSORS ? f : t, s.nbytes, g, G);
+          if (EMIT) {
+            const Emit em = emits[i];
+            if (em.len != 0)
+              copy_piece(reinterpret_cast<uint8_t*>(em.out), (TO_TENSORS ? f : t) + em.begin, em.len, g, G);
+          }
           if (VERIFY) {   // the piece's span of the stream, padding included, in aligned vectors
             const uint32_t nvec = (s.nbytes + s.pad) >> 4;
             for (uint32_t v = g; v < nvec; v += G) ck.add(ld16_cached(f + (size_t)v * 16u), v);
@@ -509,6 +514,7 @@ int launch_ring(RingMode mode, const RingLaunch& a, void* stream) {
     case kRingToFlat: return launch_ring_t<false, false, false, false>(a, stream);
     case kRingToTensors: return launch_ring_t<false, true, false, false>(a, stream);
     case kRingToTensorsVerify: return launch_ring_t<false, true, true, false>(a, stream);
+    case kRingToTensorsVerifyEmit: return launch_ring_t<false, true, true, true>(a, stream);
   }
   return (int)cudaErrorInvalidValue;
 }

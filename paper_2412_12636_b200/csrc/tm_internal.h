@@ -89,7 +89,8 @@ enum RingMode {
   kRingPackEmit,      // the same, and every piece's emit span also goes to its shard output
   kRingToFlat,        // tensors -> flat buffer (shard extract)
   kRingToTensors,     // flat buffer -> tensors (unpack, shard insert)
-  kRingToTensorsVerify  // unpack that also accumulates the checksums of the stream as read
+  kRingToTensorsVerify,  // unpack that also accumulates the checksums of the stream as read
+  kRingToTensorsVerifyEmit  // the same, and every piece's emit span also goes to its shard output
 };
 struct RingLaunch {
   const Seg* d_segs = nullptr;

@@ -62,6 +62,12 @@ class RoleMover:
         binding.tm_state_pack_emit(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
                                    None if checksums is None else checksums.data_ptr(), _stream_handle(stream))
 
+    def unpack_emit(self, buckets: torch.Tensor, checksums: torch.Tensor,
+                    stream: Optional[torch.cuda.Stream] = None) -> None:
+        """unpack + verify + the attached shards from one read of the received buckets."""
+        binding.tm_state_unpack_emit(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
+                                     checksums.data_ptr(), _stream_handle(stream))
+
     def unpack(self, buckets: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
         binding.tm_state_unpack(self.plan, buckets.data_ptr(), buckets.numel() * buckets.element_size(),
                                 _stream_handle(stream))

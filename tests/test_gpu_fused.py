@@ -273,3 +273,55 @@ def test_step_captured_in_a_cuda_graph_replays_exactly(oracle_mod):
             sub = [host[i] for i in idx]
             assert np.array_equal(out.cpu().numpy(), oracle_mod.shard(sub, [h.size for h in sub], 4, cfg.shard_r, cfg.shard_D))
     assert mover.status() == 0 and unmover.status() == 0 and sp.status() == 0
+
+
+@pytest.mark.parametrize("case", ["cfg0", "adv", "adv-ranges"])
+def test_unpack_emit_gives_tensors_checksums_and_shards_from_one_read(oracle_mod, case):
+    """The joiner's fused form: one launch over the received buckets scatters the tensors, recomputes
+    the checksums of what arrived and fills the flat shard buffers."""
+    if case == "cfg0":
+        cfg = layouts.role_config(0)
+        state = layouts.materialize(cfg, "cuda")
+        P = len(cfg.model)
+        planes, r, D, B = [(P, P), (2 * P, P), (3 * P, P)], 1, 2, cfg.bucket_bytes
+    else:
+        state, planes = _adversarial_by_elem_size(600, 18, seed=23)      # destinations at 2-byte-granular addresses
+        r, D, B = 5, 7, 1 << 20
+    host = G.host_tensors(state)
+    exp_stream, exp_cks = oracle_mod.pack(host, B)
+    exp_shards = _expected_shards(oracle_mod, host, state, planes, r, D)
+    received = torch.from_numpy(exp_stream).cuda()
+    received[7] ^= 0x40 if exp_stream.size > 7 else 0                     # damaged on the way: checksums must show it
+    exp_received = oracle_mod.checksum(received.cpu().numpy(), B)
+    target = layouts.blank_like(state)
+    outs = [G.guarded(e.size + 16) for e in exp_shards]
+    flats = [o[1][2 * p:2 * p + e.size] for p, (o, e) in enumerate(zip(outs, exp_shards))]
+    got = torch.zeros(exp_cks.size, dtype=torch.int64, device="cuda")
+    per = exp_cks.size if case != "adv-ranges" else 3
+    first, launches = 0, binding.tm_launch_count()
+    while first < exp_cks.size:
+        m = RoleMover(target.descs(), B, first_bucket=first, n_buckets=per) if case == "adv-ranges" else \
+            RoleMover(target.descs(), B)
+        m.attach_shards(planes, r, D, outs=flats)
+        lo = m.plan.stream_begin
+        m.unpack_emit(received[lo:lo + m.total_bytes], got[first:first + m.n_buckets])
+        torch.cuda.synchronize()
+        assert m.status() == 0
+        first += per
+    assert binding.tm_launch_count() == launches + -(-exp_cks.size // per)
+    assert np.array_equal(G.u64(got), exp_received) and not np.array_equal(exp_received, exp_cks)
+    damaged = oracle_mod.unpack(received.cpu().numpy(), [h.size for h in host])
+    if target.arena is not None:
+        exp_arena = np.full(target.arena.numel(), 0xA5, dtype=np.uint8)
+        for t, h in zip(target.tensors, damaged):
+            o = t.data_ptr() - target.arena.data_ptr()
+            exp_arena[o:o + h.size] = h
+        assert np.array_equal(target.arena.cpu().numpy(), exp_arena)
+    else:
+        for k, h in enumerate(damaged):
+            assert np.array_equal(target.host_bytes(k), h)
+    exp_from_received = _expected_shards(oracle_mod, damaged, state, planes, r, D)
+    for p, ((whole, _), f, e) in enumerate(zip(outs, flats, exp_from_received)):
+        assert np.array_equal(f.cpu().numpy(), e), G._first_diff(f.cpu().numpy(), e)
+        assert bool((whole[:G.GUARD + 2 * p] == G.GUARD_BYTE).all())
+        assert bool((whole[G.GUARD + 2 * p + e.size:] == G.GUARD_BYTE).all())

@@ -104,3 +104,14 @@ def test_transfer_reports_failure_when_damage_persists(oracle_mod):
     # the context is fine afterwards
     tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), cfg.bucket_bytes, 5, 2)
     _check_receiver(oracle_mod, state, target, tx, rx, cfg.bucket_bytes)
+
+
+@pytest.mark.parametrize("seed,B,per_wave,n_slots", [(0, 256, 1, 2), (1, 768, 5, 3), (2, 512, 2, 1), (3, 4096, 3, 2)])
+def test_loopback_transfer_tiny_buckets_and_odd_sizes(oracle_mod, seed, B, per_wave, n_slots):
+    # sub-vector tensors at 2-byte-granular addresses, buckets of a few hundred bytes, many waves
+    specs = layouts.odd_specs(seed, n_tensors=6 + seed)
+    state = layouts.materialize_adversarial(specs, "cuda", seed=seed)
+    target = layouts.blank_like(state)
+    tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), B, per_wave, n_slots)
+    assert rx.stats["rounds"] == 1 and tx.n_waves == -(-tx.n_buckets // per_wave)
+    _check_receiver(oracle_mod, state, target, tx, rx, B)

@@ -359,3 +359,30 @@ def test_plan_refuses_sizes_whose_sum_could_wrap(lib):
     with pytest.raises(binding.TmError) as e:
         binding.tm_shard_workspace(big, 0, 2)
     assert e.value.status == binding.TM_ERR_ARG
+
+
+def test_transfer_endpoint_geometry_and_validation(lib, oracle_mod):
+    """tm_xfer_create / tm_xfer_query are host-only: waves, slot and ring sizes follow from the
+    oracle's layout; bad geometry is refused."""
+    rng = np.random.default_rng(77)
+    sizes, descs = _random_role(rng)
+    B = 4096
+    _, T, nb = oracle_mod.layout(sizes, B)
+    arr = binding.make_descs(descs)
+    for per_wave, n_slots in ((1, 1), (3, 2), (nb + 5, 4)):
+        h = ctypes.c_void_p()
+        assert lib.tm_xfer_create(arr, len(arr), B, per_wave, n_slots, ctypes.byref(h)) == binding.TM_OK
+        nw, sb, rb, wb, nbk = ctypes.c_uint32(), ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+        assert lib.tm_xfer_query(h, ctypes.byref(nw), ctypes.byref(sb), ctypes.byref(rb), ctypes.byref(wb), ctypes.byref(nbk)) == 0
+        assert (nw.value, sb.value, rb.value, nbk.value) == (-(-nb // per_wave), per_wave * B, n_slots * per_wave * B, nb)
+        assert wb.value % 256 == 0 and wb.value >= 512 * nw.value
+        # not bound yet: running a side is refused, nothing is launched
+        t = binding.TmTransport()
+        assert lib.tm_xfer_send(h, ctypes.byref(t), None, None, 3, None) == binding.TM_ERR_STATE
+        lib.tm_xfer_destroy(h)
+    h = ctypes.c_void_p()
+    for per_wave, n_slots, code in ((0, 2, binding.TM_ERR_ARG), (2, 0, binding.TM_ERR_ARG), (2, 65, binding.TM_ERR_ARG),
+                                    (1 << 40, 2, binding.TM_ERR_ARG)):
+        assert lib.tm_xfer_create(arr, len(arr), B, per_wave, n_slots, ctypes.byref(h)) == code and not h.value
+    assert lib.tm_xfer_create(arr, len(arr), 100, 2, 2, ctypes.byref(h)) == binding.TM_ERR_ALIGN
+    assert lib.tm_xfer_create(None, 0, B, 2, 2, ctypes.byref(h)) == binding.TM_ERR_ARG
