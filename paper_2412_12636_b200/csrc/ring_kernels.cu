@@ -35,7 +35,10 @@ constexpr int kRingStages = 3;
 constexpr uint32_t kStageBytes = 32 * 1024;
 constexpr uint32_t kStageVectors = kStageBytes / 16;
 constexpr uint32_t kStageStride = kStageBytes + 128;   // room for the one extra vector of a shifted source
-constexpr int kConsWarps = 8;
+#ifndef TM_CONS_WARPS
+#define TM_CONS_WARPS 8
+#endif
+constexpr int kConsWarps = TM_CONS_WARPS;
 constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kRingThreads = kConsThreads + 64;     // + one producer warp + one store warp
 constexpr uint32_t kBulkMinVectors = 128;           // pieces below 2 KiB are not worth a stage
