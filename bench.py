@@ -294,7 +294,8 @@ def run_reference(args) -> None:
 class RoleBench:
     """One role on the current GPU with every buffer the step needs."""
 
-    def __init__(self, workload: str, prepared=None, layers: Optional[int] = None, shard: Optional[Tuple[int, int]] = None):
+    def __init__(self, workload: str, prepared=None, layers: Optional[int] = None, shard: Optional[Tuple[int, int]] = None,
+                 tensors: int = 20_000):
         from paper_2412_12636_b200 import layouts
         from paper_2412_12636_b200.mover import MultiShardExtractor, RoleMover, ShardExtractor, ShardPlanMover
         if prepared is not None:      # (RoleState, bucket_bytes, r, D): a wave of a larger role
@@ -302,8 +303,8 @@ class RoleBench:
             self.name = self.state.name
             planes = [self.state.elem_size_indices(4)]
         elif workload == "cfg4lite":
-            self.state = layouts.materialize_adversarial(layouts.adversarial_specs(20_000), "cuda")
-            self.name, self.bucket_bytes, self.shard_r, self.shard_D = "adversarial-20000", layouts.ADVERSARIAL_BUCKET, 29, 64
+            self.state = layouts.materialize_adversarial(layouts.adversarial_specs(tensors), "cuda")
+            self.name, self.bucket_bytes, self.shard_r, self.shard_D = f"adversarial-{tensors}", layouts.ADVERSARIAL_BUCKET, 29, 64
             planes = [self.state.elem_size_indices(4)]
         else:
             cfg = layouts.role_config(WORKLOADS[workload], layers=layers)
@@ -613,7 +614,7 @@ def run_ours(args) -> None:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     shard = tuple(int(x) for x in args.shard.split(",")) if args.shard else None
-    role = RoleBench(args.workload, layers=args.layers, shard=shard)
+    role = RoleBench(args.workload, layers=args.layers, shard=shard, tensors=args.tensors)
     for _ in range(max(args.warmup, 3)):
         role.one_step()
     torch.cuda.synchronize()
@@ -878,6 +879,8 @@ def main() -> None:
     ap.add_argument("--layers", type=int, default=None,
                     help="reduce cfg0..cfg3 to their first LAYERS transformer layers: a small, self-ending case "
                          "(a few GB, still far larger than the L2) for profiler captures")
+    ap.add_argument("--tensors", type=int, default=20_000,
+                    help="cfg4lite: number of tensors of the adversarial set (2000 gives a 2.6 GB case for profiler captures)")
     ap.add_argument("--shard", default="", help="R,D: override the workload's shard rank and count (cfg0..cfg3)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="only the kernels of the step and of the fused calls: no transfer pipeline, host tier, "

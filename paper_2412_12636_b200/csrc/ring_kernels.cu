@@ -3,9 +3,14 @@
 // ring of stages guarded by mbarriers.  When source and destination are both 16-byte aligned the
 // stage goes straight back out, shared memory -> global, with a bulk store issued by one store
 // thread, and the eight consumer warps only read the stage to accumulate the checksum.  When the
-// source sits at a 2-byte-granular address the consumers re-align the stage in registers and write
-// 16-byte vectors themselves.  The producer runs ahead across piece and item boundaries, so the
-// loads of the next pieces are in flight while the current one is consumed.
+// source sits at a 2-byte-granular address the consumers re-align the stage in registers.  In pack
+// and unpack they write the aligned vectors into a second ring of "out" stages in shared memory and
+// the store thread sends those out with bulk stores as well (bulk stores keep DRAM busier than
+// 16-byte stores from registers: +1.5 % on a role whose tensors are all misaligned).  The plain
+// gather into a flat buffer (shard extract: short launches, where the extra hand-over costs more
+// than it gains) stores the re-aligned vectors from registers.  The producer runs ahead across
+// piece and item boundaries, so the loads of the next pieces are in flight while the current one is
+// consumed.
 //
 // Misaligned sources cost no extra global traffic here: the producer fetches the aligned superset
 // of the source span (one extra 16-byte vector per stage) and the consumers shift in registers.
@@ -35,6 +40,7 @@ constexpr int kRingStages = 3;
 constexpr uint32_t kStageBytes = 32 * 1024;
 constexpr uint32_t kStageVectors = kStageBytes / 16;
 constexpr uint32_t kStageStride = kStageBytes + 128;   // room for the one extra vector of a shifted source
+constexpr int kOutStages = 3;                          // re-aligned stages waiting for their bulk store
 #ifndef TM_CONS_WARPS
 #define TM_CONS_WARPS 8
 #endif
@@ -141,8 +147,13 @@ __device__ __forceinline__ bool plan_bulk(const Seg& s, uint8_t* flat, BulkPlan&
 struct RingShared {
   uint64_t full[kRingStages];
   uint64_t empty[kRingStages];
+  uint64_t out_full[kOutStages];    // the consumer warps have written a re-aligned stage
+  uint64_t out_empty[kOutStages];   // its bulk store has finished reading it
   int abort_flag;
 };
+
+// Makes this thread's ordinary shared-memory writes visible to the bulk-copy engine.
+__device__ __forceinline__ void fence_smem_for_bulk() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void raise_timeout(int* status, RingShared* sh) {
   if (status != nullptr) atomicExch(status, (int)TM_ERR_TIMEOUT);
@@ -212,11 +223,18 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       mbar_init(&sh.full[s], 1);
       mbar_init(&sh.empty[s], kConsWarps + 1);   // consumer warps + the store thread
     }
+    for (int s = 0; s < kOutStages; ++s) {
+      mbar_init(&sh.out_full[s], kConsWarps);
+      mbar_init(&sh.out_empty[s], 1);
+    }
     sh.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   volatile int* abort_flag = &sh.abort_flag;
+  // re-aligned stages leave through the out ring (bulk stores) in pack and unpack, from registers otherwise
+  constexpr bool RESTAGE = PACK || TO_TENSORS;
+  uint8_t* const out_ring = ring + (size_t)kRingStages * kStageStride;
 
   if (warp == kConsWarps) {
     // ---------------- producer: one thread issues every bulk load of this block, in item order
@@ -264,10 +282,12 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
   }
 
   if (warp == kConsWarps + 1) {
-    // ---------------- store thread: sends aligned stages back out with bulk stores, in item order
+    // ---------------- store thread: sends every stage back out with bulk stores, in item order —
+    // straight from the load stage when source and destination are aligned alike, else from the out
+    // stage the consumers have re-aligned it into
     if (lane != 0) return;
-    uint32_t stage = 0, phase = 0;
-    int pending = -1;   // stage whose bulk store may still be reading shared memory
+    uint32_t stage = 0, phase = 0, ostage = 0, ophase = 0;
+    uint64_t* pending = nullptr;   // barrier to release once the newest bulk store has finished reading shared memory
     bool ok = true;
     for (uint32_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
       const uint32_t first = item_first[item];
@@ -281,29 +301,45 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
           ok = false;
           break;
         }
+        uint32_t cnt = p.nfull - t * p.V;
+        if (cnt > p.V) cnt = p.V;
+        const uint8_t* from;
+        uint64_t* release;
         if (p.straight) {
-          uint32_t cnt = p.nfull - t * p.V;
-          if (cnt > p.V) cnt = p.V;
-          bulk_s2g(p.dst + (size_t)t * p.V * 16u, ring + (size_t)stage * kStageStride, cnt * 16u);
-          bulk_commit();
-          if (pending >= 0) {
-            bulk_wait_read<1>();
-            mbar_arrive(&sh.empty[pending]);
-          }
-          pending = (int)stage;
+          from = ring + (size_t)stage * kStageStride;
+          release = &sh.empty[stage];
         } else {
-          if (pending >= 0) {
-            bulk_wait_read<0>();
-            mbar_arrive(&sh.empty[pending]);
-            pending = -1;
+          mbar_arrive(&sh.empty[stage]);   // the consumers read this stage; the store thread does not
+          if (!RESTAGE) {                  // ... and write its data themselves
+            if (pending != nullptr) {
+              bulk_wait_read<0>();
+              mbar_arrive(pending);
+              pending = nullptr;
+            }
+            if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
+            continue;
           }
-          mbar_arrive(&sh.empty[stage]);   // the consumers write this stage's data themselves
+          if (!mbar_wait(&sh.out_full[ostage], ophase, abort_flag, wait_limit_ns)) {
+            raise_timeout(status, &sh);
+            ok = false;
+            break;
+          }
+          from = out_ring + (size_t)ostage * kStageBytes;
+          release = &sh.out_empty[ostage];
+          if (++ostage == kOutStages) { ostage = 0; ophase ^= 1u; }
         }
+        bulk_s2g(p.dst + (size_t)t * p.V * 16u, from, cnt * 16u);
+        bulk_commit();
+        if (pending != nullptr) {
+          bulk_wait_read<1>();
+          mbar_arrive(pending);
+        }
+        pending = release;
         if (++stage == kRingStages) { stage = 0; phase ^= 1u; }
       }
     }
     bulk_wait_read<0>();
-    if (pending >= 0) mbar_arrive(&sh.empty[pending]);
+    if (pending != nullptr) mbar_arrive(pending);
     bulk_wait_all();
     return;
   }
@@ -313,7 +349,7 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
   Cksum ck;
   u64 total = 0;
   uint32_t cur = 0xffffffffu;
-  uint32_t stage = 0, phase = 0;
+  uint32_t stage = 0, phase = 0, ostage = 0, ophase = 0;
   bool ok = true;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t first = item_first[item], last = item_first[item + 1];
@@ -392,22 +428,36 @@ ring_kernel(const Seg* __restrict__ segs, const uint32_t* __restrict__ item_firs
       const uint8_t* stage_base = ring + (size_t)stage * kStageStride;
       const uint4* sp = reinterpret_cast<const uint4*>(stage_base);
       const uint32_t vbase = t * p.V;
-      uint8_t* d = p.dst + (size_t)vbase * 16u;
       // VERIFY: the stream piece starts 256-byte aligned, so stage vector v is stream vector vbase + v
       if (p.straight) {
         if (PACK || VERIFY) {   // the store thread moves the data; only the checksum is left to do
 #pragma unroll 4
           for (uint32_t v = c; v < cnt; v += kConsThreads) ck.add(sp[v], vbase + v);
         }
+      } else if (!RESTAGE) {
+        uint8_t* d = p.dst + (size_t)vbase * 16u;
+#pragma unroll 2
+        for (uint32_t v = c; v < cnt; v += kConsThreads) st16(d + (size_t)v * 16u, shift_pair(sp[v], sp[v + 1], ws, bs));
       } else {
+        // re-align into an out stage whose previous bulk store has finished reading it
+        if (!__all_sync(0xffffffffu, mbar_wait(&sh.out_empty[ostage], ophase ^ 1u, abort_flag, wait_limit_ns))) {
+          raise_timeout(status, &sh);
+          ok = false;
+          break;
+        }
+        uint4* op = reinterpret_cast<uint4*>(out_ring + (size_t)ostage * kStageBytes);
 #pragma unroll 2
         for (uint32_t v = c; v < cnt; v += kConsThreads) {
           const uint4 lo = sp[v];
           const uint4 x = shift_pair(lo, sp[v + 1], ws, bs);
-          st16(d + (size_t)v * 16u, x);
+          op[v] = x;
           if (PACK) ck.add(x, vbase + v);
           if (VERIFY) ck.add(lo, vbase + v);
         }
+        fence_smem_for_bulk();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.out_full[ostage]);
+        if (++ostage == kOutStages) { ostage = 0; ophase ^= 1u; }
       }
       if (EMIT && em.len != 0) {
         // this stage holds piece bytes [s_lo, s_hi), byte b at stage_base + a + (b - s_lo)
@@ -496,7 +546,7 @@ static int launch_ring_t(const RingLaunch& a, void* stream) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return (int)e;
-  const size_t smem = (size_t)kRingStages * kStageStride;
+  const size_t smem = (size_t)kRingStages * kStageStride + ((PACK || TO_TENSORS) ? (size_t)kOutStages * kStageBytes : 0);
   auto kernel = ring_kernel<PACK, TO_TENSORS, VERIFY, EMIT>;
   e = ensure_smem(kernel, smem, dev, attr_done);
   if (e != cudaSuccess) return (int)e;

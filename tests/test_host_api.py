@@ -386,3 +386,53 @@ def test_transfer_endpoint_geometry_and_validation(lib, oracle_mod):
         assert lib.tm_xfer_create(arr, len(arr), B, per_wave, n_slots, ctypes.byref(h)) == code and not h.value
     assert lib.tm_xfer_create(arr, len(arr), 100, 2, 2, ctypes.byref(h)) == binding.TM_ERR_ALIGN
     assert lib.tm_xfer_create(None, 0, B, 2, 2, ctypes.byref(h)) == binding.TM_ERR_ARG
+
+
+def test_shard_plan_and_attach_validation_without_a_device(lib):
+    """Argument checks of the reusable shard plan and of the shard attachment run before any device
+    work, so they can be exercised with no workspace at all."""
+    plane = _descs([4096, 8192, 4096], elem=4)                       # three fp32 tensors, 16 MiB apart
+    sp = binding.ShardPlan([plane], 0, 2)
+    assert sp.elems == [2048] and sp.out_bytes == [8192]
+    far = FAKE + (1 << 40)
+    cases = [
+        ([far + 1], [8192], binding.TM_ERR_ALIGN),                   # odd output address
+        ([far], [8191], binding.TM_ERR_CAPACITY),                    # output too small
+        ([plane[0][0] + 64], [1 << 20], binding.TM_ERR_OVERLAP),     # output inside a source tensor
+        ([0], [8192], binding.TM_ERR_ARG),                           # missing output
+    ]
+    for flats, caps, code in cases:
+        with pytest.raises(binding.TmError) as e:
+            sp.bind(flats, caps, None, 0, 0)
+        assert e.value.status == code, (flats, caps)
+    two = binding.ShardPlan([plane, _descs([4096], elem=2, base=FAKE + (1 << 36))], 1, 2)
+    with pytest.raises(binding.TmError) as e:                        # the two outputs overlap each other
+        two.bind([far, far + 100], [1 << 20, 1 << 20], None, 0, 0)
+    assert e.value.status == binding.TM_ERR_OVERLAP
+    with pytest.raises(binding.TmError) as e:                        # never bound: nothing to run
+        binding.ShardPlan([plane], 0, 2).extract(0)
+    assert e.value.status == binding.TM_ERR_STATE
+    for bad in ((0, 0), (2, 2)):
+        with pytest.raises(binding.TmError) as e:
+            binding.ShardPlan([plane], *bad)
+        assert e.value.status == binding.TM_ERR_RANK
+    with pytest.raises(binding.TmError) as e:                        # mixed element sizes inside one plane
+        binding.ShardPlan([plane + _descs([64], elem=2, base=FAKE + (1 << 37))], 0, 2)
+    assert e.value.status == binding.TM_ERR_DTYPE
+
+    plan = binding.Plan(plane, 4096)
+    ok_out, cap = [far], [1 << 20]
+    for planes, outs, caps, code in (
+            ([(0, 3)], [plane[1][0]], cap, binding.TM_ERR_OVERLAP),  # shard output on top of a tensor
+            ([(0, 3)], [far + 1], cap, binding.TM_ERR_ALIGN),
+            ([(0, 3)], ok_out, [100], binding.TM_ERR_CAPACITY),
+            ([(0, 4)], ok_out, cap, binding.TM_ERR_ARG),             # plane runs past the descriptors
+            ([(0, 2), (1, 2)], [far, far + (1 << 30)], [1 << 20] * 2, binding.TM_ERR_ARG),   # planes overlap
+            ([(0, 0)], ok_out, cap, binding.TM_ERR_ARG)):            # empty plane
+        with pytest.raises(binding.TmError) as e:
+            binding.tm_plan_attach_shards(plan, planes, 0, 2, outs, caps, None, 0, 0)
+        assert e.value.status == code, (planes, outs)
+    elems, need = binding.tm_plan_attach_shards(plan, [(0, 3)], 1, 2, ok_out, cap, None, 0, 0)
+    assert elems == [2048] and need > plan.workspace_bytes
+    emits = plan.emits()
+    assert int(emits["len"].sum()) == 8192                           # the shard's bytes, each named once
