@@ -40,7 +40,10 @@ constexpr int kRingStages = 3;
 constexpr uint32_t kStageBytes = 32 * 1024;
 constexpr uint32_t kStageVectors = kStageBytes / 16;
 constexpr uint32_t kStageStride = kStageBytes + 128;   // room for the one extra vector of a shifted source
-constexpr int kOutStages = 3;                          // re-aligned stages waiting for their bulk store
+#ifndef TM_OUT_STAGES
+#define TM_OUT_STAGES 3
+#endif
+constexpr int kOutStages = TM_OUT_STAGES;              // re-aligned stages waiting for their bulk store
 #ifndef TM_CONS_WARPS
 #define TM_CONS_WARPS 8
 #endif
