@@ -227,6 +227,44 @@ def test_ring_kernel_waits_made_to_expire_leave_everything_in_bounds(oracle_mod)
     torch.cuda.synchronize()
     assert normal.status() == 0 and G.guards_intact(whole, normal.total_bytes)
     assert np.array_equal(buckets.cpu().numpy(), exp_stream) and np.array_equal(G.u64(cks), exp_cks)
+    # the same for the receiving side and the shard gather, on a layout whose tensors are misaligned
+    # (re-aligned stages, out ring): targets live in one arena, so a stray write would show
+    adv = layouts.materialize_adversarial(layouts.adversarial_specs(300, max_log2=17), "cuda", seed=41)
+    host = G.host_tensors(adv)
+    stream_a, cks_a = oracle_mod.pack(host, 1 << 20)
+    received = torch.from_numpy(stream_a).cuda()
+    target = layouts.blank_like(adv)
+    idx = adv.elem_size_indices(4)
+    exp_shard = oracle_mod.shard([host[i] for i in idx], [host[i].size for i in idx], 4, 3, 5)
+    sw, sout = G.guarded(exp_shard.size)
+    try:
+        binding.tm_options_set(wait_limit_ns=1)
+        hasty_rx = RoleMover(target.descs(), 1 << 20)
+        hasty_sp = ShardPlanMover([adv.descs_of(idx)], 3, 5, flats=[sout])
+    finally:
+        binding.tm_options_set()
+    got = hasty_rx.alloc_checksums()
+    seen = set()
+    for _ in range(5):
+        hasty_rx.unpack_verify(received, got)
+        hasty_sp.extract()
+        seen |= {hasty_rx.status(), hasty_sp.status()}
+        assert G.guards_intact(sw, exp_shard.size)
+    assert seen <= {0, binding.TM_ERR_TIMEOUT}
+    covered = torch.zeros(target.arena.numel(), dtype=torch.bool, device="cuda")
+    for t, spec in zip(target.tensors, target.specs):
+        o = t.data_ptr() - target.arena.data_ptr()
+        covered[o:o + spec.nbytes] = True
+    assert bool((target.arena[~covered] == 0xA5).all())          # nothing written between the tensors
+    rx = RoleMover(target.descs(), 1 << 20)
+    rx.unpack_verify(received, got)
+    sp = ShardPlanMover([adv.descs_of(idx)], 3, 5, flats=[sout])
+    sp.extract()
+    torch.cuda.synchronize()
+    assert rx.status() == 0 and sp.status() == 0 and np.array_equal(G.u64(got), cks_a)
+    for k in range(len(host)):
+        assert np.array_equal(target.host_bytes(k), host[k])
+    assert np.array_equal(sout.cpu().numpy(), exp_shard) and G.guards_intact(sw, exp_shard.size)
 
 
 def test_step_captured_in_a_cuda_graph_replays_exactly(oracle_mod):
