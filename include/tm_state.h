@@ -114,7 +114,7 @@ typedef struct tm_options {
   uint64_t cksum_tile_bytes;   /* tile of the stand-alone checksum kernel; multiple of 256; default 256 KiB */
   uint64_t wait_limit_ns;      /* bound of every device-side wait of the ring kernels; 1 .. 5e9; default 2e9 */
   uint32_t group_max;          /* piece budget of a shared item; 1 .. 1024; default 64 */
-  uint32_t ring_ctas_per_sm;   /* persistent blocks per SM of the ring kernels (96 KiB of shared memory each); 1 .. 2; default 1 */
+  uint32_t ring_ctas_per_sm;   /* persistent blocks per SM of the ring kernels (96 KiB of shared memory each, 192 KiB in pack and unpack, where a second block does not fit); 1 .. 2; default 1 */
   uint32_t ctas_per_sm;        /* persistent blocks per SM of the checksum kernel; 1 .. 8; default 4 */
   uint32_t reserved;           /* must be 0 */
 } tm_options;
