@@ -132,7 +132,10 @@ int tm_options_set(const tm_options* in);
  * `descs` is copied; it may be freed after the call.  *out receives a plan to be released with
  * tm_plan_destroy.  Errors: TM_ERR_ARG (NULL, n_desc == 0, nbytes == 0, nbytes % elem_size != 0,
  * bucket_bytes == 0 or > 2^35, nbytes > 2^46, n_desc > 2^24, T > 2^56), TM_ERR_DTYPE, TM_ERR_ALIGN
- * (odd ptr, bucket_bytes % 256 != 0), TM_ERR_CAPACITY (out of host memory). */
+ * (odd ptr, bucket_bytes % 256 != 0), TM_ERR_CAPACITY (out of host memory, or a work list of more than
+ * 2^24 pieces — 4 TiB of stream at the default piece size, far less with tiny buckets; such a role is
+ * planned in ranges).  The same piece limit applies to a bound shard plan and to all waves of a
+ * transfer endpoint together. */
 int tm_plan_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_plan** out);
 
 /* Plan for a run of whole buckets of the same stream — the unit in which a role travels through a

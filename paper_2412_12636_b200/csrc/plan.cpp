@@ -103,15 +103,12 @@ using tms::Seg;
 
 static inline uint64_t align256(uint64_t x) { return (x + 255) & ~(uint64_t)255; }
 
-// Validates the descriptors, computes off_k / T / n_buckets of the complete stream and the
-// pack / unpack work list of the plan's range (all buckets unless `ranged`).
-int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, bool ranged,
-                  uint64_t first_bucket, uint64_t n_buckets) {
+// Validates the descriptors and computes off_k, T and the bucket count of the complete stream.
+int tm_layout_build(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_layout* out) {
   if (descs == nullptr || n_desc == 0 || bucket_bytes == 0) return TM_ERR_ARG;
   if (bucket_bytes > (1ull << 35)) return TM_ERR_ARG;
   if (bucket_bytes % 256 != 0) return TM_ERR_ALIGN;
   if (n_desc > tms::kMaxDescs) return TM_ERR_ARG;
-  if (ranged && n_buckets == 0) return TM_ERR_ARG;
   uint64_t sum = 0;   // running stream length; bounded inside the loop, so it cannot wrap
   for (uint64_t k = 0; k < n_desc; ++k) {
     const tm_desc& d = descs[k];
@@ -122,12 +119,31 @@ int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bu
     sum = align256(sum) + d.nbytes;
     if (sum > tms::kMaxTotalBytes) return TM_ERR_ARG;
   }
+  out->offsets.resize(n_desc);
+  uint64_t pos = 0;
+  for (uint64_t k = 0; k < n_desc; ++k) {
+    out->offsets[k] = align256(pos);
+    pos = out->offsets[k] + descs[k].nbytes;
+  }
+  out->bucket_bytes = bucket_bytes;
+  out->whole_bytes = align256(pos);
+  out->whole_buckets = (out->whole_bytes + bucket_bytes - 1) / bucket_bytes;
+  return TM_OK;
+}
+
+// Cuts the part of the stream that the plan covers (all buckets unless `ranged`) into the pack /
+// unpack work list.  `cursor` (may be NULL): in, a descriptor index at or before the first tensor
+// that reaches into the range; out, the last tensor that does — consecutive ranges of one role are
+// then cut in one pass over the descriptors.  The list is refused (TM_ERR_CAPACITY) before any of it
+// is built when it would exceed kMaxPieces pieces.
+int tm_plan_fill(tm_plan* p, const tm_desc* descs, uint64_t n_desc, const tm_layout& lay, bool ranged,
+                 uint64_t first_bucket, uint64_t n_buckets, uint64_t* cursor) {
+  if (ranged && n_buckets == 0) return TM_ERR_ARG;
+  const uint64_t bucket_bytes = lay.bucket_bytes;
   p->opt = tms::tuning();
-  p->descs.assign(descs, descs + n_desc);
   p->bucket_bytes = bucket_bytes;
-  p->offsets.resize(n_desc);
-  p->whole_bytes = align256(sum);
-  p->whole_buckets = (p->whole_bytes + bucket_bytes - 1) / bucket_bytes;
+  p->whole_bytes = lay.whole_bytes;
+  p->whole_buckets = lay.whole_buckets;
   uint64_t range_lo = 0, range_hi = p->whole_bytes;
   if (ranged) {
     if (first_bucket >= p->whole_buckets) return TM_ERR_ARG;
@@ -144,19 +160,30 @@ int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bu
   p->total_bytes = range_hi - range_lo;
 
   const uint64_t chunk = p->opt.chunk_bytes;
+  // first tensor that reaches into the range
+  uint64_t k0 = (cursor != nullptr && *cursor < n_desc) ? *cursor : 0;
+  while (k0 > 0 && lay.offsets[k0] > range_lo) --k0;
+  while (k0 < n_desc && lay.offsets[k0] + descs[k0].nbytes <= range_lo) ++k0;
+  // upper bound on the pieces: a part of n bytes is cut at chunk ends and at bucket ends
+  uint64_t bound = 0;
+  for (uint64_t k = k0; k < n_desc && lay.offsets[k] < range_hi; ++k) {
+    const uint64_t a = std::max(lay.offsets[k], range_lo), b = std::min(lay.offsets[k] + descs[k].nbytes, range_hi);
+    if (a < b) bound += (b - a) / chunk + (b - a) / bucket_bytes + 2;
+    if (bound > tms::kMaxPieces) return TM_ERR_CAPACITY;
+  }
+
   tms::WorkListBuilder builder(&p->work, p->opt);
   p->piece_desc.clear();
   p->parts.clear();
   p->box_lo = ~0ull;
   p->box_hi = 0;
-  uint64_t pos = 0;
-  for (uint64_t k = 0; k < n_desc; ++k) {
-    const uint64_t off = align256(pos);
-    p->offsets[k] = off;
+  uint64_t last = k0;
+  for (uint64_t k = k0; k < n_desc && lay.offsets[k] < range_hi; ++k) {
+    const uint64_t off = lay.offsets[k];
     const uint64_t end = off + descs[k].nbytes;
-    pos = end;
     const uint64_t a = std::max(off, range_lo), b = std::min(end, range_hi);
     if (a >= b) continue;                                   // the tensor has no byte in the range
+    last = k;
     uint64_t tensor = (uint64_t)(uintptr_t)descs[k].ptr + (a - off);
     p->parts.push_back(tm_part{tensor, b - a});
     p->box_lo = std::min(p->box_lo, tensor);
@@ -186,9 +213,22 @@ int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bu
     }
   }
   builder.finish();
+  if (cursor != nullptr) *cursor = last;
   if (p->box_lo == ~0ull) p->box_lo = 0;
-  if (p->work.segs.size() >= (1ull << 32) - (1u << 20)) return TM_ERR_ARG;   // piece and item indices are 32-bit
   p->ws_layout = tms::workspace_layout(p->work.segs.size(), p->work.n_items());
+  return TM_OK;
+}
+
+// A plan that owns its copy of the descriptors and offsets (what the public plan calls need).
+int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, bool ranged,
+                  uint64_t first_bucket, uint64_t n_buckets) {
+  tm_layout lay;
+  int rc = tm_layout_build(descs, n_desc, bucket_bytes, &lay);
+  if (rc != TM_OK) return rc;
+  rc = tm_plan_fill(p, descs, n_desc, lay, ranged, first_bucket, n_buckets, nullptr);
+  if (rc != TM_OK) return rc;
+  p->descs.assign(descs, descs + n_desc);
+  p->offsets = std::move(lay.offsets);
   return TM_OK;
 }
 

@@ -90,6 +90,11 @@ int plan_bind(tm_shard_plan* sp, void* const* d_flats, const uint64_t* capacitie
       if (flats[q].second != 0 && tms::ranges_overlap(flats[p].first, flats[p].second, flats[q].first, flats[q].second))
         return TM_ERR_OVERLAP;
   }
+  uint64_t bound = 0;
+  for (uint32_t p = 0; p < n_planes; ++p) {
+    if (flats[p].second != 0) bound += max_pieces(sp, p);
+    if (bound > tms::kMaxPieces) return TM_ERR_CAPACITY;   // refused before any of the list is built
+  }
   tms::WorkList wl;
   tms::WorkListBuilder builder(&wl, sp->opt);
   const tm_desc* cursor = sp->descs.data();

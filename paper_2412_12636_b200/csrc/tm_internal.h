@@ -81,6 +81,9 @@ inline bool ranges_overlap(uint64_t a, uint64_t an, uint64_t b, uint64_t bn) { r
 constexpr uint64_t kMaxTensorBytes = 1ull << 46;
 constexpr uint64_t kMaxDescs = 1ull << 24;
 constexpr uint64_t kMaxTotalBytes = 1ull << 56;
+// Longest work list that is built (pieces): 16 M pieces are 512 MiB of host memory and, at the default
+// piece sizes, 4 TiB of stream or 1 TiB of shard.  Longer lists are refused before anything is allocated.
+constexpr uint64_t kMaxPieces = 1ull << 24;
 
 // ---- kernel launchers.  Each returns a cudaError_t as int. -----------------------------------
 // What a ring launch does with the pieces of its list.
@@ -172,7 +175,16 @@ struct tm_shard_plan {
   int targets_disjoint = 0;
 };
 
+// Layout of a complete stream: off_k of every descriptor, T and the bucket count.
+struct tm_layout {
+  std::vector<uint64_t> offsets;
+  uint64_t bucket_bytes = 0, whole_bytes = 0, whole_buckets = 0;
+};
+
 // planner (plan.cpp)
+int tm_layout_build(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, tm_layout* out);
+int tm_plan_fill(tm_plan* p, const tm_desc* descs, uint64_t n_desc, const tm_layout& lay, bool ranged,
+                 uint64_t first_bucket, uint64_t n_buckets, uint64_t* cursor);
 int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, bool ranged,
                   uint64_t first_bucket, uint64_t n_buckets);
 int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);

@@ -299,18 +299,29 @@ int tm_xfer_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes,
       x->bucket_bytes = bucket_bytes;
       x->per_wave = buckets_per_wave;
       x->n_slots = n_slots;
-      uint64_t first = 0;
-      do {
+      // one pass over the descriptors for the layout, one more for all waves together: the wave plans
+      // hold their pieces only, not a copy of the role's descriptor list each
+      tm_layout lay;
+      rc = tm_layout_build(descs, n_desc, bucket_bytes, &lay);
+      if (rc == TM_OK) {
+        x->n_buckets = lay.whole_buckets;
+        if ((lay.whole_buckets + buckets_per_wave - 1) / buckets_per_wave > (1u << 20)) rc = TM_ERR_ARG;   // more waves than any ring is driven with
+        // all waves together hold the pieces of the whole stream: refuse an over-long list before building any
+        const uint64_t bound = lay.whole_bytes / tms::tuning().chunk_bytes + lay.whole_bytes / bucket_bytes;
+        if (rc == TM_OK && bound > tms::kMaxPieces) rc = TM_ERR_CAPACITY;
+      }
+      uint64_t first = 0, cursor = 0, pieces = 0;
+      while (rc == TM_OK && first < x->n_buckets) {
         tm_plan* p = new tm_plan();
         x->waves.push_back(p);
-        rc = tm_plan_build(p, descs, n_desc, bucket_bytes, /*ranged=*/true, first, buckets_per_wave);
+        rc = tm_plan_fill(p, descs, n_desc, lay, /*ranged=*/true, first, buckets_per_wave, &cursor);
         if (rc != TM_OK) break;
-        x->n_buckets = p->whole_buckets;
+        pieces += p->work.segs.size();
+        if (pieces > tms::kMaxPieces) rc = TM_ERR_CAPACITY;
         x->ws_off.push_back(x->workspace_bytes);
         x->workspace_bytes += p->ws_layout.total;
         first += buckets_per_wave;
-        if (x->waves.size() > (1u << 20)) rc = TM_ERR_ARG;   // more waves than any ring would be driven with
-      } while (rc == TM_OK && first < x->n_buckets);
+      }
     } catch (...) {
       delete x;
       throw;

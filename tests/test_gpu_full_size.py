@@ -377,3 +377,26 @@ def test_tensor_beyond_4_gib_and_word_index_beyond_2_31():
     assert ex.extract(out) == ex.hi - ex.lo
     torch.cuda.synchronize()
     assert torch.equal(out.view(torch.int64), t[ex.lo:ex.hi])
+    del out
+    torch.cuda.empty_cache()
+    # the fused and the ranged forms at the same sizes: stream offsets, range offsets and shard outputs
+    # all beyond 32 bits.  Pack + checksums + the shard from one read ...
+    B = 1 << 30
+    mover = RoleMover(state.descs(), B)
+    (shard_out,) = mover.attach_shards([(0, 1)], 2, 3)
+    buckets, cks = mover.alloc_buckets(), mover.alloc_checksums()
+    mover.pack_emit(buckets, cks)
+    torch.cuda.synchronize()
+    assert mover.status() == 0
+    assert torch.equal(buckets.view(torch.int64), t) and torch.equal(shard_out.view(torch.int64), t[ex.lo:ex.hi])
+    words = [min(B // 8, n - j * (B // 8)) for j in range(mover.n_buckets)]
+    assert [int(x) for x in G.u64(cks)] == [(c * w * w) % M64 for w in words]
+    del buckets, shard_out, mover
+    torch.cuda.empty_cache()
+    # ... and the same tensor sent through a ring of two 2 GiB slots per side
+    from paper_2412_12636_b200 import transfer
+    back = torch.zeros_like(t)
+    tx, rx, _ = transfer.loopback_transfer(state.descs(), [(back.data_ptr(), 8 * n, 8, layouts.PLANE_OTHER)], B, 2, 2)
+    assert tx.n_waves == 9 and rx.stats["rounds"] == 1 and rx.stats["bad_buckets"] == 0
+    assert torch.equal(back, t)
+    assert [int(x) for x in G.u64(rx.checksums)] == [(c * w * w) % M64 for w in words]

@@ -361,6 +361,35 @@ def test_plan_refuses_sizes_whose_sum_could_wrap(lib):
     assert e.value.status == binding.TM_ERR_ARG
 
 
+def test_lists_too_long_to_build_are_refused_before_any_allocation(lib):
+    """Sizes that pass the per-tensor limits but would need hundreds of millions of pieces (a 64 TiB
+    tensor in 256-byte buckets) are refused at once with TM_ERR_CAPACITY instead of exhausting host
+    memory while the list grows."""
+    import time
+    huge = [(FAKE, 1 << 46, 4, 1)]
+    t0 = time.perf_counter()
+    for B in (256, 1 << 20, 1 << 35):
+        with pytest.raises(binding.TmError) as e:
+            binding.Plan(huge, B)
+        assert e.value.status == binding.TM_ERR_CAPACITY
+        with pytest.raises(binding.TmError) as e:
+            binding.Plan(huge, B, 0, 1 << 30)
+        assert e.value.status == binding.TM_ERR_CAPACITY
+    small_range = binding.Plan(huge, 1 << 30, 5, 2)               # two buckets of it are a reasonable plan
+    assert small_range.total_bytes == 2 << 30 and small_range.stream_begin == 5 << 30
+    sp = binding.ShardPlan([huge], 0, 2)
+    assert sp.out_bytes == [1 << 45]
+    with pytest.raises(binding.TmError) as e:
+        sp.bind([FAKE + (1 << 60)], [1 << 62], None, 0, 0)
+    assert e.value.status == binding.TM_ERR_CAPACITY
+    h = ctypes.c_void_p()
+    arr = binding.make_descs(huge)
+    assert lib.tm_xfer_create(arr, 1, 1 << 20, 1, 2, ctypes.byref(h)) == binding.TM_ERR_ARG          # over 2^20 waves
+    assert lib.tm_xfer_create(arr, 1, 1 << 30, 1024, 2, ctypes.byref(h)) == binding.TM_ERR_CAPACITY  # 64 waves, too many pieces
+    assert not h.value
+    assert time.perf_counter() - t0 < 5.0
+
+
 def test_transfer_endpoint_geometry_and_validation(lib, oracle_mod):
     """tm_xfer_create / tm_xfer_query are host-only: waves, slot and ring sizes follow from the
     oracle's layout; bad geometry is refused."""
@@ -436,3 +465,51 @@ def test_shard_plan_and_attach_validation_without_a_device(lib):
     assert elems == [2048] and need > plan.workspace_bytes
     emits = plan.emits()
     assert int(emits["len"].sum()) == 8192                           # the shard's bytes, each named once
+
+
+def test_random_arguments_never_crash_the_host_entry_points(lib, oracle_mod):
+    """Random, mostly unreasonable arguments to every host-only entry point: the call either succeeds
+    with a layout that agrees with the oracle, or returns a negative status — it never crashes, and
+    never reports sizes that wrapped around."""
+    rng = np.random.default_rng(2024)
+    sizes_pool = [0, 1, 2, 6, 254, 256, 258, 4096, (1 << 20) + 2, 1 << 33, (1 << 46), (1 << 46) + 8, (1 << 63)]
+    for trial in range(300):
+        n = int(rng.integers(0, 6))
+        descs = []
+        for k in range(n):
+            e = int(rng.choice([2, 4, 8, 8, 4, 2, 3, 0, 16]))
+            nb = int(rng.choice(sizes_pool))
+            ptr = int(rng.choice([FAKE + (k << 47), FAKE + (k << 47) + 1, 0, FAKE]))   # FAKE twice: overlapping tensors
+            descs.append((ptr, nb, e, 0))
+        B = int(rng.choice([0, 100, 256, 768, 1 << 20, 1 << 35, (1 << 35) + 256]))
+        first, count = int(rng.integers(0, 5)), int(rng.integers(0, 4))
+        ok_sizes = all(d[1] > 0 and d[2] in (2, 4, 8) and d[1] % d[2] == 0 and d[1] <= (1 << 46) and d[0] and d[0] % 2 == 0
+                       for d in descs)
+        try:
+            plan = binding.Plan(descs, B, first, count) if trial % 2 else binding.Plan(descs, B)
+        except binding.TmError as e:
+            assert e.status < 0
+            plan = None
+        if plan is not None:
+            assert n > 0 and ok_sizes and B % 256 == 0 and 0 < B <= (1 << 35)
+            off, T, nbk = oracle_mod.layout([d[1] for d in descs], B)
+            assert plan.offsets() == [int(x) for x in off] and (plan.whole_bytes, plan.whole_buckets) == (T, nbk)
+            assert plan.total_bytes <= T and plan.n_buckets <= nbk
+            pieces, items = plan.pieces()
+            assert int(pieces["nbytes"].astype(np.uint64).sum() + pieces["pad"].astype(np.uint64).sum()) == plan.total_bytes
+        r, D = int(rng.integers(0, 4)), int(rng.integers(0, 4))
+        try:
+            sp = binding.ShardPlan([descs], r, D) if n else None
+            if sp is not None:
+                e0 = descs[0][2]
+                assert ok_sizes and all(d[2] == e0 for d in descs) and D > 0 and r < D
+                N = sum(d[1] for d in descs) // e0
+                assert sp.elems == [oracle_mod.shard_bounds(N, r, D)[1] - oracle_mod.shard_bounds(N, r, D)[0]]
+                try:
+                    sp.bind([FAKE + (1 << 60)], [1 << 62], None, 0, 0)        # host-only: the list is only built
+                    p2, _, _ = sp.pieces()
+                    assert int(p2["nbytes"].astype(np.uint64).sum()) == sp.out_bytes[0]
+                except (binding.TmError, MemoryError) as e:
+                    assert not isinstance(e, binding.TmError) or e.status < 0
+        except binding.TmError as e:
+            assert e.status < 0
