@@ -363,3 +363,45 @@ def test_unpack_emit_gives_tensors_checksums_and_shards_from_one_read(oracle_mod
         assert np.array_equal(f.cpu().numpy(), e), G._first_diff(f.cpu().numpy(), e)
         assert bool((whole[:G.GUARD + 2 * p] == G.GUARD_BYTE).all())
         assert bool((whole[G.GUARD + 2 * p + e.size:] == G.GUARD_BYTE).all())
+
+
+@pytest.mark.parametrize("opts", [
+    dict(chunk_bytes=8192, shard_chunk_bytes=4096, small_bytes=1024, group_bytes=4096, group_max=4),
+    dict(ring_ctas_per_sm=2, ctas_per_sm=8, cksum_tile_bytes=4096),
+    dict(chunk_bytes=1 << 30, shard_chunk_bytes=1 << 30, small_bytes=1 << 20, group_bytes=1 << 22, group_max=1024),
+])
+def test_results_do_not_depend_on_the_tuning_values(oracle_mod, opts):
+    """The tuning values change how the work is cut and spread, never what is computed: with tiny
+    pieces, with huge pieces and with two blocks per SM every result still equals the oracle's."""
+    state, planes = _adversarial_by_elem_size(500, 17, seed=29)
+    B = 1 << 19
+    host = G.host_tensors(state)
+    exp_stream, exp_cks = oracle_mod.pack(host, B)
+    exp_shards = _expected_shards(oracle_mod, host, state, planes, 3, 5)
+    try:
+        binding.tm_options_set(**opts)
+        mover = RoleMover(state.descs(), B)
+        outs = mover.attach_shards(planes, 3, 5)
+        target = layouts.blank_like(state)
+        unmover = RoleMover(target.descs(), B)
+        sp = ShardPlanMover([state.descs_of(list(range(f, f + c))) for f, c in planes], 3, 5)
+        whole, buckets = G.guarded(mover.total_bytes)
+        fused, alone, got = mover.alloc_checksums(), mover.alloc_checksums(), mover.alloc_checksums()
+        mover.pack_emit(buckets, fused)
+        mover.checksum(buckets, alone)            # reads the tile size in force now
+    finally:
+        binding.tm_options_set()
+    unmover.unpack_verify(buckets, got)
+    sp.extract()
+    torch.cuda.synchronize()
+    assert mover.status() == 0 and unmover.status() == 0 and sp.status() == 0 and G.guards_intact(whole, mover.total_bytes)
+    assert np.array_equal(buckets.cpu().numpy(), exp_stream)
+    for c in (fused, alone, got):
+        assert np.array_equal(G.u64(c), exp_cks)
+    for out, flat, e in zip(outs, sp.flats, exp_shards):
+        assert np.array_equal(out.cpu().numpy(), e) and np.array_equal(flat.cpu().numpy(), e)
+    exp_arena = np.full(target.arena.numel(), 0xA5, dtype=np.uint8)
+    for t, h in zip(target.tensors, host):
+        o = t.data_ptr() - target.arena.data_ptr()
+        exp_arena[o:o + h.size] = h
+    assert np.array_equal(target.arena.cpu().numpy(), exp_arena)
