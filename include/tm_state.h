@@ -442,6 +442,18 @@ int tm_xfer_query(const tm_xfer* x, uint32_t* n_waves, uint64_t* slot_bytes, uin
  * sender's values as received; NULL on the sender).  Creates the events that order slot hand-overs. */
 int tm_xfer_bind(tm_xfer* x, void* d_ring, uint64_t ring_bytes, void* d_workspace, uint64_t workspace_bytes,
                  uint64_t* d_checksums, uint64_t* d_peer_checksums, void* stream);
+/* Optional: shards filled during the transfer.  Planes, r, D, outputs and the size query (d_workspace
+ * == NULL) as for tm_plan_attach_shards, applied to every wave; afterwards the sender packs with
+ * tm_state_pack_emit and the receiver unpacks with tm_state_unpack_emit, so that a joiner under the
+ * distributed optimizer has its flat slices of master weights, m and v when the last wave has been
+ * verified (§7 "State Synchronization"), from the same read that scatters the tensors.  A wave that is
+ * sent again rewrites its part of the shards.  Call after tm_xfer_bind; d_workspace is further
+ * caller-owned scratch (256-byte aligned) that must stay untouched while the endpoint is in use. */
+int tm_xfer_attach_shards(tm_xfer* x, const uint64_t* plane_first_desc, const uint64_t* plane_n_desc, uint32_t n_planes,
+                          uint32_t r, uint32_t D, void* const* d_outs, const uint64_t* out_capacities,
+                          uint64_t* out_elems, void* d_workspace, uint64_t workspace_bytes,
+                          uint64_t* workspace_needed, void* stream);
+
 /* Run one side to the end.  Packing (unpacking) is enqueued on the first stream, the transport's
  * send (recv) on the second; the two must differ for the steps to overlap.  The calls block the host
  * until the last round's report has been exchanged; the receiver's tensors are complete when

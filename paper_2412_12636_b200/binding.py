@@ -42,6 +42,7 @@ SIGNATURES = {
     "tm_xfer_create": (_int, [_p, _u64, _u64, _u64, _u32, _p]),
     "tm_xfer_query": (_int, [_p, _p, _p, _p, _p, _p]),
     "tm_xfer_bind": (_int, [_p, _p, _u64, _p, _u64, _p, _p, _p]),
+    "tm_xfer_attach_shards": (_int, [_p, _p, _p, _u32, _u32, _u32, _p, _p, _p, _p, _u64, _p, _p]),
     "tm_xfer_send": (_int, [_p, _p, _p, _p, _u32, _p]),
     "tm_xfer_receive": (_int, [_p, _p, _p, _p, _u32, _p]),
     "tm_xfer_destroy": (None, [_p]),

@@ -353,15 +353,18 @@ int tm_state_unpack_verify(const tm_plan* plan, const void* d_buckets, uint64_t 
   });
 }
 
-int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const uint64_t* plane_n_desc,
-                          uint32_t n_planes, uint32_t r, uint32_t D, void* const* d_outs,
-                          const uint64_t* out_capacities, uint64_t* out_elems, void* d_workspace,
-                          uint64_t workspace_bytes, uint64_t* workspace_needed, void* stream) {
+}  // extern "C"
+
+// Shard attachment for a plan whose pieces index into `descs` (the plan's own copy, or the one copy a
+// transfer endpoint keeps for all of its wave plans).
+int tm_attach_shards(tm_plan* plan, const tm_desc* descs, uint64_t n_desc, const uint64_t* plane_first_desc,
+                     const uint64_t* plane_n_desc, uint32_t n_planes, uint32_t r, uint32_t D, void* const* d_outs,
+                     const uint64_t* out_capacities, uint64_t* out_elems, void* d_workspace,
+                     uint64_t workspace_bytes, uint64_t* workspace_needed, void* stream) {
   return guarded([&]() -> int {
-    if (plan == nullptr || plane_first_desc == nullptr || plane_n_desc == nullptr || n_planes == 0)
+    if (plan == nullptr || descs == nullptr || plane_first_desc == nullptr || plane_n_desc == nullptr || n_planes == 0)
       return TM_ERR_ARG;
     if (D == 0 || r >= D) return TM_ERR_RANK;
-    const uint64_t n_desc = plan->descs.size();
     struct PlaneInfo { uint64_t first, n; uint32_t e; uint64_t lo, hi; };
     std::vector<PlaneInfo> planes(n_planes);
     uint64_t prev_end = 0;
@@ -372,7 +375,7 @@ int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const
       if (pi.n == 0 || pi.first < prev_end || pi.n > n_desc || pi.first > n_desc - pi.n) return TM_ERR_ARG;   // ascending, disjoint
       prev_end = pi.first + pi.n;
       uint64_t n_elems = 0;
-      int rc = tm_shard_validate(plan->descs.data() + pi.first, pi.n, r, D, &pi.e, &n_elems);
+      int rc = tm_shard_validate(descs + pi.first, pi.n, r, D, &pi.e, &n_elems);
       if (rc != TM_OK) return rc;
       rc = tm_bounds_u128(n_elems, r, D, &pi.lo, &pi.hi);
       if (rc != TM_OK) return rc;
@@ -405,7 +408,7 @@ int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const
       for (uint64_t k = planes[p].first; k < planes[p].first + planes[p].n; ++k) {
         desc_plane[k] = (int32_t)p;
         desc_start[k] = start;
-        start += plan->descs[k].nbytes / planes[p].e;
+        start += descs[k].nbytes / planes[p].e;
       }
     }
     // one emit record per piece: the piece's bytes that are shard elements, and where they go
@@ -418,11 +421,11 @@ int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const
       const uint32_t k = plan->piece_desc[i];
       if (desc_plane[k] < 0) continue;
       const PlaneInfo& pi = planes[desc_plane[k]];
-      const uint64_t start = desc_start[k], count = plan->descs[k].nbytes / pi.e;
+      const uint64_t start = desc_start[k], count = descs[k].nbytes / pi.e;
       const uint64_t a = std::max(pi.lo, start), b = std::min(pi.hi, start + count);
       if (a >= b) continue;
       const tms::Seg& s = plan->work.segs[i];
-      const uint64_t x = s.tensor - (uint64_t)(uintptr_t)plan->descs[k].ptr;   // piece = tensor bytes [x, x + nbytes)
+      const uint64_t x = s.tensor - (uint64_t)(uintptr_t)descs[k].ptr;   // piece = tensor bytes [x, x + nbytes)
       const uint64_t sa = (a - start) * pi.e, sb = (b - start) * pi.e;         // shard = tensor bytes [sa, sb)
       const uint64_t lo = std::max(x, sa), hi = std::min(x + s.nbytes, sb);
       if (lo >= hi) continue;
@@ -440,6 +443,17 @@ int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const
     plan->emit_outs = std::move(outs);
     return TM_OK;
   });
+}
+
+extern "C" {
+
+int tm_plan_attach_shards(tm_plan* plan, const uint64_t* plane_first_desc, const uint64_t* plane_n_desc,
+                          uint32_t n_planes, uint32_t r, uint32_t D, void* const* d_outs,
+                          const uint64_t* out_capacities, uint64_t* out_elems, void* d_workspace,
+                          uint64_t workspace_bytes, uint64_t* workspace_needed, void* stream) {
+  if (plan == nullptr) return TM_ERR_ARG;
+  return tm_attach_shards(plan, plan->descs.data(), plan->descs.size(), plane_first_desc, plane_n_desc, n_planes, r, D,
+                          d_outs, out_capacities, out_elems, d_workspace, workspace_bytes, workspace_needed, stream);
 }
 
 int tm_state_pack_emit(const tm_plan* plan, void* d_buckets, uint64_t capacity, uint64_t* d_checksums,

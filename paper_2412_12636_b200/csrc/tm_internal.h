@@ -187,6 +187,10 @@ int tm_plan_fill(tm_plan* p, const tm_desc* descs, uint64_t n_desc, const tm_lay
                  uint64_t first_bucket, uint64_t n_buckets, uint64_t* cursor);
 int tm_plan_build(tm_plan* p, const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes, bool ranged,
                   uint64_t first_bucket, uint64_t n_buckets);
+int tm_attach_shards(tm_plan* plan, const tm_desc* descs, uint64_t n_desc, const uint64_t* plane_first_desc,
+                     const uint64_t* plane_n_desc, uint32_t n_planes, uint32_t r, uint32_t D, void* const* d_outs,
+                     const uint64_t* out_capacities, uint64_t* out_elems, void* d_workspace,
+                     uint64_t workspace_bytes, uint64_t* workspace_needed, void* stream);   // api.cpp
 int tm_bounds_u128(uint64_t n_elems, uint32_t r, uint32_t D, uint64_t* lo, uint64_t* hi);
 int tm_shard_validate(const tm_desc* descs, uint64_t n_desc, uint32_t r, uint32_t D, uint32_t* elem_size,
                       uint64_t* n_elems);

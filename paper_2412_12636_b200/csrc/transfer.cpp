@@ -126,6 +126,8 @@ extern "C" int tm_xfer_run_receiver(uint32_t n_waves, uint32_t n_slots, uint32_t
 // ---- one side of a transfer on the GPU -------------------------------------------------------------
 
 struct tm_xfer {
+  std::vector<tm_desc> descs;           // the role's descriptors (one copy for all waves)
+  bool emits = false;                   // shards attached: packing / unpacking also fills them
   std::vector<tm_plan*> waves;          // one range plan per wave
   std::vector<uint64_t> ws_off;         // each plan's place in the workspace
   uint64_t bucket_bytes = 0, per_wave = 0, n_buckets = 0, slot_bytes = 0, workspace_bytes = 0;
@@ -162,7 +164,9 @@ int hook_pack(void* ctx, uint32_t wave, uint32_t slot) {
   if (check_wave(x, wave, slot) != TM_OK) return TM_ERR_ARG;
   const tm_plan* p = x->waves[wave];
   if (x->used[slot]) TM_CUDA(cudaStreamWaitEvent(x->work_stream, x->drained[slot], 0));   // the transport has read the slot
-  int rc = tm_state_pack(p, x->slot_ptr(slot), x->slot_bytes, x->d_checksums + p->first_bucket, x->work_stream);
+  int rc = x->emits
+      ? tm_state_pack_emit(p, x->slot_ptr(slot), x->slot_bytes, x->d_checksums + p->first_bucket, x->work_stream)
+      : tm_state_pack(p, x->slot_ptr(slot), x->slot_bytes, x->d_checksums + p->first_bucket, x->work_stream);
   if (rc != TM_OK) return rc;
   TM_CUDA(cudaEventRecord(x->filled[slot], x->work_stream));
   return TM_OK;
@@ -206,7 +210,9 @@ int hook_unpack_verify(void* ctx, uint32_t wave, uint32_t slot) {
   if (check_wave(x, wave, slot) != TM_OK) return TM_ERR_ARG;
   const tm_plan* p = x->waves[wave];
   TM_CUDA(cudaStreamWaitEvent(x->work_stream, x->filled[slot], 0));
-  int rc = tm_state_unpack_verify(p, x->slot_ptr(slot), p->total_bytes, x->d_checksums + p->first_bucket, x->work_stream);
+  int rc = x->emits
+      ? tm_state_unpack_emit(p, x->slot_ptr(slot), p->total_bytes, x->d_checksums + p->first_bucket, x->work_stream)
+      : tm_state_unpack_verify(p, x->slot_ptr(slot), p->total_bytes, x->d_checksums + p->first_bucket, x->work_stream);
   if (rc != TM_OK) return rc;
   TM_CUDA(cudaEventRecord(x->drained[slot], x->work_stream));
   x->used[slot] = 1;
@@ -296,6 +302,7 @@ int tm_xfer_create(const tm_desc* descs, uint64_t n_desc, uint64_t bucket_bytes,
     tm_xfer* x = new tm_xfer();
     int rc = TM_OK;
     try {
+      if (descs != nullptr && n_desc <= tms::kMaxDescs) x->descs.assign(descs, descs + n_desc);
       x->bucket_bytes = bucket_bytes;
       x->per_wave = buckets_per_wave;
       x->n_slots = n_slots;
@@ -373,6 +380,38 @@ int tm_xfer_bind(tm_xfer* x, void* d_ring, uint64_t ring_bytes, void* d_workspac
     x->d_ring = (uint8_t*)d_ring;
     x->d_checksums = d_checksums;
     x->d_peer = d_peer_checksums;
+    return TM_OK;
+  });
+}
+
+int tm_xfer_attach_shards(tm_xfer* x, const uint64_t* plane_first_desc, const uint64_t* plane_n_desc, uint32_t n_planes,
+                          uint32_t r, uint32_t D, void* const* d_outs, const uint64_t* out_capacities,
+                          uint64_t* out_elems, void* d_workspace, uint64_t workspace_bytes,
+                          uint64_t* workspace_needed, void* stream) {
+  if (x == nullptr) return TM_ERR_ARG;
+  if (((uintptr_t)d_workspace & 255) != 0) return TM_ERR_ALIGN;
+  return guarded([&]() -> int {
+    // size pass: every wave's list with its emit records
+    uint64_t need = 0;
+    std::vector<uint64_t> off(x->waves.size());
+    for (size_t w = 0; w < x->waves.size(); ++w) {
+      uint64_t n = 0;
+      int rc = tm_attach_shards(x->waves[w], x->descs.data(), x->descs.size(), plane_first_desc, plane_n_desc, n_planes, r, D,
+                                nullptr, nullptr, w == 0 ? out_elems : nullptr, nullptr, 0, &n, stream);
+      if (rc != TM_OK) return rc;
+      off[w] = need;
+      need += n;
+    }
+    if (workspace_needed != nullptr) *workspace_needed = need;
+    if (d_workspace == nullptr) return TM_OK;
+    if (workspace_bytes < need) return TM_ERR_CAPACITY;
+    for (size_t w = 0; w < x->waves.size(); ++w) {
+      const uint64_t span = (w + 1 < off.size() ? off[w + 1] : need) - off[w];
+      int rc = tm_attach_shards(x->waves[w], x->descs.data(), x->descs.size(), plane_first_desc, plane_n_desc, n_planes, r, D,
+                                d_outs, out_capacities, nullptr, (uint8_t*)d_workspace + off[w], span, nullptr, stream);
+      if (rc != TM_OK) return rc;
+    }
+    x->emits = true;
     return TM_OK;
   });
 }

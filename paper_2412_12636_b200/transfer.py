@@ -49,6 +49,25 @@ class Endpoint:
                               self.peer_checksums.data_ptr() if receiver else None, _stream_handle(stream)),
                "tm_xfer_bind")
 
+    def attach_shards(self, planes: Sequence[Tuple[int, int]], r: int, D: int, elem_sizes: Sequence[int], stream=None):
+        """Shards filled during the transfer: `planes` = (first descriptor, count) runs of the role,
+        `elem_sizes` their element sizes.  Allocates and returns the flat outputs (uint8 tensors)."""
+        L = binding.load_library()
+        n = len(planes)
+        first = (_u64 * n)(*[p[0] for p in planes])
+        count = (_u64 * n)(*[p[1] for p in planes])
+        got, need = (_u64 * n)(), _u64()
+        _check(L.tm_xfer_attach_shards(self._h, first, count, n, r, D, None, None, got, None, 0, ctypes.byref(need), 0),
+               "tm_xfer_attach_shards")
+        sizes = [g * e for g, e in zip(got, elem_sizes)]
+        self.shard_outs = [torch.empty(max(s, 1), dtype=torch.uint8, device=self.device)[:s] for s in sizes]
+        self.shard_workspace = torch.empty(max(need.value, 256), dtype=torch.uint8, device=self.device)
+        outs = (_p * n)(*[o.data_ptr() for o in self.shard_outs])
+        caps = (_u64 * n)(*sizes)
+        _check(L.tm_xfer_attach_shards(self._h, first, count, n, r, D, outs, caps, None, self.shard_workspace.data_ptr(),
+                                       self.shard_workspace.numel(), None, _stream_handle(stream)), "tm_xfer_attach_shards")
+        return self.shard_outs
+
     def run(self, transport: "binding.TmTransport", work_stream, wire_stream, max_rounds: int = 3) -> Dict[str, int]:
         """Sender: packs on `work_stream`, sends on `wire_stream`.  Receiver: unpacks + verifies on
         `work_stream`, receives on `wire_stream`.  Blocks until the last report has been exchanged;
@@ -268,15 +287,20 @@ def run_protocol(sender: bool, n_waves: int, n_slots: int, max_rounds: int, **st
 
 
 def loopback_transfer(send_descs, recv_descs, bucket_bytes: int, buckets_per_wave: int, n_slots: int,
-                      max_rounds: int = 3, after_recv: Optional[Callable] = None, device="cuda"):
+                      max_rounds: int = 3, after_recv: Optional[Callable] = None, device="cuda",
+                      recv_shards: Optional[Tuple[Sequence[Tuple[int, int]], int, int]] = None):
     """Moves a role from `send_descs` to `recv_descs` on one GPU: two endpoints, the loopback
     transport, four streams, the receiver in a second host thread.  `after_recv(rx, wave, d_slot,
     nbytes, stream)` is called on the receiving side after every recv has been enqueued (tests damage
-    the arrived slot there).  Returns (sender endpoint, receiver endpoint, elapsed device milliseconds
+    the arrived slot there).  `recv_shards` = (planes, r, D) makes the receiver fill its flat shards
+    while it unpacks (rx.shard_outs).  Returns (sender endpoint, receiver endpoint, elapsed device milliseconds
     between the first pack and the last unpack)."""
     import threading
     tx = Endpoint(send_descs, bucket_bytes, buckets_per_wave, n_slots, receiver=False, device=device)
     rx = Endpoint(recv_descs, bucket_bytes, buckets_per_wave, n_slots, receiver=True, device=device)
+    if recv_shards is not None:      # (planes, r, D): the receiver also fills its flat shards
+        planes, r, D = recv_shards
+        rx.attach_shards(planes, r, D, [recv_descs[f][2] for f, _ in planes])
     lb = Loopback()
     rx_transport = lb.transport
     if after_recv is not None:

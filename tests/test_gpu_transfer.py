@@ -115,3 +115,36 @@ def test_loopback_transfer_tiny_buckets_and_odd_sizes(oracle_mod, seed, B, per_w
     tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), B, per_wave, n_slots)
     assert rx.stats["rounds"] == 1 and tx.n_waves == -(-tx.n_buckets // per_wave)
     _check_receiver(oracle_mod, state, target, tx, rx, B)
+
+
+@pytest.mark.parametrize("case", ["cfg0", "adversarial"])
+def test_receiver_fills_its_shards_while_the_role_arrives(oracle_mod, case):
+    """With shards attached to the receiving endpoint, every wave's unpack also writes its part of the
+    joiner's flat slices; a wave damaged in flight first writes damaged shard bytes, and its repeat
+    repairs them along with the tensors."""
+    if case == "cfg0":
+        cfg = layouts.role_config(0)
+        state = layouts.materialize(cfg, "cuda")
+        P = len(cfg.model)
+        planes, r, D, B, per_wave = [(P, P), (2 * P, P), (3 * P, P)], 1, 2, cfg.bucket_bytes, 3
+    else:
+        specs = sorted(layouts.adversarial_specs(600, max_log2=17), key=lambda s: s.elem_size)
+        state = layouts.materialize_adversarial(specs, "cuda", seed=19)
+        planes, k = [], 0
+        for e in (2, 4, 8):
+            c = sum(1 for s in specs if s.elem_size == e)
+            planes.append((k, c))
+            k += c
+        r, D, B, per_wave = 4, 9, 1 << 18, 4
+    target = layouts.blank_like(state)
+    host = G.host_tensors(state)
+    n_waves = -(-oracle_mod.layout([h.size for h in host], B)[2] // per_wave)
+    hits = {(1, w): 1000 + 37 * w for w in range(0, n_waves, 2)}        # every second wave arrives damaged once
+    tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), B, per_wave, 2, max_rounds=3,
+                                           after_recv=_flip_on_host(hits, {}), recv_shards=(planes, r, D))
+    assert rx.stats["rounds"] == 2 and rx.stats["waves_again"] == len(hits)
+    _check_receiver(oracle_mod, state, target, tx, rx, B)
+    for (first, count), out in zip(planes, rx.shard_outs):
+        sub = host[first:first + count]
+        expect = oracle_mod.shard(sub, [h.size for h in sub], state.specs[first].elem_size, r, D)
+        assert np.array_equal(out.cpu().numpy(), expect), (first, count)
