@@ -8,8 +8,10 @@ attribute does, and fails loudly if it has not been built.
 """
 
 _BINDING_NAMES = (
-    "Plan", "TmError", "tm_state_pack", "tm_state_unpack", "tm_shard_extract", "tm_shard_insert", "tm_shard_extract_static", "tm_checksum",
-    "tm_shard_bounds", "tm_shard_workspace", "tm_launch_count", "load_library", "make_descs",
+    "Plan", "ShardPlan", "TmError", "tm_state_pack", "tm_state_unpack", "tm_state_unpack_verify", "tm_state_pack_emit",
+    "tm_state_unpack_emit", "tm_plan_attach_shards", "tm_shard_extract", "tm_shard_extract_planes", "tm_shard_insert",
+    "tm_shard_extract_static", "tm_checksum", "tm_shard_bounds", "tm_shard_workspace", "tm_options_get", "tm_options_set",
+    "tm_launch_count", "load_library", "make_descs",
 )
 
 

@@ -1,11 +1,11 @@
-"""Processing a role whose state does not fit one GPU next to its packed copy, in waves.
+"""Which tensors of a role to materialise for a run of whole buckets.
 
-Buckets are independent units (each has its own checksum, word index restarting at 0), so a role
-can be packed as consecutive runs of descriptors, each run covering a whole number of buckets of the
-complete stream.  A tensor that straddles the cut between two runs is split at the bucket boundary
-into two descriptors; the cut lies on a multiple of the bucket size, hence of 256, so both halves
-keep the alignment rules and the concatenation of the runs' streams is the complete stream, byte
-for byte and checksum for checksum.
+The library cuts a role into runs of whole buckets itself (tm_plan_create_range, tm_xfer_*).  A role
+whose state does not fit one GPU at all — the 200 000-tensor adversarial set is about 257 GB — also
+needs its *inputs* generated run by run; this module tells the input generators which tensors, and
+which byte range of a tensor that straddles a cut, belong to each run.  Buckets are independent
+units (each has its own checksum, word index restarting at 0), and a cut lies on a multiple of the
+bucket size, hence of 256, so the runs' streams and checksum lists concatenate to the complete ones.
 
 `offsets` are the stream offsets of the complete descriptor list as reported by the planner
 (`Plan.offsets()`); this module only compares them with multiples of the bucket size.
