@@ -3,9 +3,10 @@ library's tm_xfer objects and transports.  The protocol (slot assignment, rounds
 waves) and every data-path step run inside the library; this module allocates the ring, scratch and
 checksum arrays with PyTorch and marshals arguments.
 
-Transports: `Loopback` (both sides in one process on one GPU, the library's own), and
+Transports: `Loopback` (both sides in one process on one GPU, the library's own),
 `TorchDistTransport`, which moves whole slots with torch.distributed send / recv (NCCL between two
-GPUs; gloo between two CPU processes in the protocol tests).
+GPUs; gloo between two CPU processes in the protocol tests), and `HostRelayTransport`, which relays
+slots through pinned host memory between two processes (also two that share one GPU).
 """
 from __future__ import annotations
 
@@ -215,6 +216,51 @@ class TorchDistTransport:
             for i in range(count):
                 waves[i] = int(msg[1 + i].item())
             n[0] = count
+            return 0
+        except Exception:
+            return binding.TM_ERR_TRANSPORT
+
+
+class HostRelayTransport(TorchDistTransport):
+    """Slots travel through pinned host memory: the sender copies a slot device -> host on the given
+    stream, waits for it and sends the host buffer with torch.distributed (any backend that moves CPU
+    tensors, e.g. gloo); the receiver receives into pinned host memory and copies host -> device on
+    its stream.  For two processes without a GPU-to-GPU link between them — also two processes that
+    share one GPU.  `device_owners` are the endpoint's device tensors the raw addresses point into
+    (ring, checksums, peer checksums); `damage(wave, host_slot)` (optional) may alter the host copy
+    before it is sent."""
+
+    def __init__(self, peer: int, device_owners: Sequence[torch.Tensor], slot_bytes: int, max_checksums: int,
+                 group=None, damage: Optional[Callable] = None):
+        self.host_slot = torch.empty(slot_bytes, dtype=torch.uint8, pin_memory=True)
+        self.host_cks = torch.empty(max_checksums, dtype=torch.int64, pin_memory=True)
+        self.damage = damage
+        super().__init__(peer, list(device_owners), report_device="cpu", group=group)
+
+    def _send(self, ctx, wave, d_slot, nbytes, d_cks, n_cks, stream):
+        try:
+            st = torch.cuda.ExternalStream(stream) if stream else torch.cuda.current_stream()
+            with torch.cuda.stream(st):
+                self.host_slot[:nbytes].copy_(self._view(d_slot, nbytes, torch.uint8), non_blocking=True)
+                self.host_cks[:n_cks].copy_(self._view(d_cks, 8 * n_cks, torch.int64), non_blocking=True)
+            st.synchronize()
+            if self.damage is not None:
+                self.damage(wave, self.host_slot[:nbytes])
+            self.dist.send(self.host_slot[:nbytes], self.peer, group=self.group, tag=2 * wave)
+            self.dist.send(self.host_cks[:n_cks], self.peer, group=self.group, tag=2 * wave + 1)
+            return 0
+        except Exception:
+            return binding.TM_ERR_TRANSPORT
+
+    def _recv(self, ctx, wave, d_slot, nbytes, d_cks, n_cks, stream):
+        try:
+            st = torch.cuda.ExternalStream(stream) if stream else torch.cuda.current_stream()
+            st.synchronize()      # the previous copies out of the host staging buffers have finished
+            self.dist.recv(self.host_slot[:nbytes], self.peer, group=self.group, tag=2 * wave)
+            self.dist.recv(self.host_cks[:n_cks], self.peer, group=self.group, tag=2 * wave + 1)
+            with torch.cuda.stream(st):
+                self._view(d_slot, nbytes, torch.uint8).copy_(self.host_slot[:nbytes], non_blocking=True)
+                self._view(d_cks, 8 * n_cks, torch.int64).copy_(self.host_cks[:n_cks], non_blocking=True)
             return 0
         except Exception:
             return binding.TM_ERR_TRANSPORT

@@ -148,3 +148,75 @@ def test_receiver_fills_its_shards_while_the_role_arrives(oracle_mod, case):
         sub = host[first:first + count]
         expect = oracle_mod.shard(sub, [h.size for h in sub], state.specs[first].elem_size, r, D)
         assert np.array_equal(out.cpu().numpy(), expect), (first, count)
+
+
+TWO_PROCESS_WORKER = r"""
+import os, sys, json
+sys.path.insert(0, os.environ["TM_ROOT"])
+sys.path.insert(0, os.path.join(os.environ["TM_ROOT"], "tests"))
+import numpy as np, torch, torch.distributed as dist
+import oracle
+from paper_2412_12636_b200 import binding, layouts, transfer
+dist.init_process_group("gloo")
+rank = dist.get_rank()
+torch.cuda.set_device(0)
+binding.load_library()
+cfg = layouts.role_config(0)
+B, per_wave, n_slots = cfg.bucket_bytes, 3, 2
+state = layouts.materialize(cfg, "cuda")                     # same seed in both processes
+host = [state.host_bytes(k) for k in range(len(state.tensors))]
+_, exp_cks = oracle.pack(host, B)
+streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+if rank == 0:                                                # the leaver's process
+    ep = transfer.Endpoint(state.descs(), B, per_wave, n_slots, receiver=False)
+    sent = {}
+    def damage(wave, host_slot):                             # wave 4 leaves damaged the first time
+        sent[wave] = sent.get(wave, 0) + 1
+        if wave == 4 and sent[wave] == 1:
+            host_slot[4321] ^= 0x08
+    tr = transfer.HostRelayTransport(1, [ep.ring, ep.checksums], ep.slot_bytes, per_wave, damage=damage)
+    stats = ep.run(tr.transport, streams[0], streams[1], 3)
+    result = {"rank": 0, "stats": stats, "checksums_ok": bool(np.array_equal(ep.checksums.cpu().numpy().view(np.uint64), exp_cks))}
+else:                                                        # the joiner's process
+    target = layouts.blank_like(state)
+    ep = transfer.Endpoint(target.descs(), B, per_wave, n_slots, receiver=True)
+    tr = transfer.HostRelayTransport(0, [ep.ring, ep.checksums, ep.peer_checksums], ep.slot_bytes, per_wave)
+    stats = ep.run(tr.transport, streams[0], streams[1], 3)
+    torch.cuda.synchronize()
+    result = {"rank": 1, "stats": stats,
+              "tensors_ok": all(np.array_equal(target.host_bytes(k), host[k]) for k in range(len(host))),
+              "checksums_ok": bool(np.array_equal(ep.checksums.cpu().numpy().view(np.uint64), exp_cks))}
+dist.barrier()
+print(json.dumps(result))
+dist.destroy_process_group()
+"""
+
+
+def test_leaver_and_joiner_in_two_processes(tmp_path):
+    """The two sides as two processes (gloo ranks 0 and 1) that share this GPU: each runs its endpoint
+    with the library's kernels, slots cross between the processes through pinned host memory.  No
+    kernel of one process waits for the other — only the host threads block in send / recv — so the
+    processes may time-share the device.  One wave is damaged on the way and must be repaired."""
+    import json, os, socket, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "worker.py"
+    script.write_text(TWO_PROCESS_WORKER)
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, TM_ROOT=root, RANK=str(rank), LOCAL_RANK="0", WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        out, err = p.communicate(timeout=300)
+        assert p.returncode == 0, err[-3000:]
+        outs.append(json.loads(out.strip().splitlines()[-1]))
+    tx, rx = sorted(outs, key=lambda o: o["rank"])
+    for o in (tx, rx):
+        assert o["stats"]["rounds"] == 2 and o["stats"]["waves"] == 9 + 1 and o["stats"]["waves_again"] == 1
+        assert o["checksums_ok"]
+    assert rx["tensors_ok"] and rx["stats"]["bad_buckets"] == 1 and rx["stats"]["first_bad_bucket"] == 12
