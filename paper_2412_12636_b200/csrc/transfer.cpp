@@ -435,8 +435,11 @@ void tm_xfer_destroy(tm_xfer* x) { delete x; }
 struct tm_loopback {
   std::mutex m;
   std::condition_variable cv;
-  // one posted receive at a time
+  // one posted receive at a time; `posts` and `taken` count the receives posted and the receives whose
+  // stream has been made to wait for the sender's copy (a sender waits for "its" receive by number: the
+  // receiver may already have posted the next one when the sender wakes up)
   bool posted = false, matched = false;
+  uint64_t posts = 0, taken = 0;
   int match_rc = TM_OK;
   uint32_t wave = 0;
   void* d_slot = nullptr;
@@ -471,12 +474,14 @@ int lb_recv(void* ctx, uint32_t wave, void* d_slot, uint64_t nbytes, uint64_t* d
   lb->n_cks = n_cks;
   lb->matched = false;
   lb->posted = true;
+  lb->posts += 1;
   lb->cv.notify_all();
   const bool met = lb->cv.wait_for(lock, kPartnerTimeout, [&] { return lb->matched; });
   int rc = met ? lb->match_rc : TM_ERR_TRANSPORT;
   if (rc == TM_OK && cudaStreamWaitEvent((cudaStream_t)stream, lb->data_ready, 0) != cudaSuccess) rc = TM_ERR_CUDA;
   lb->posted = false;
   lb->matched = false;
+  lb->taken += 1;
   lb->cv.notify_all();
   return rc;
 }
@@ -499,9 +504,10 @@ int lb_send(void* ctx, uint32_t wave, const void* d_slot, uint64_t nbytes, const
   }
   lb->match_rc = rc;
   lb->matched = true;
+  const uint64_t mine = lb->posts;
   lb->cv.notify_all();
   // data_ready must not be recorded again before the receiver has made its stream wait on this record
-  if (!lb->cv.wait_for(lock, kPartnerTimeout, [&] { return !lb->posted; })) return TM_ERR_TRANSPORT;
+  if (!lb->cv.wait_for(lock, kPartnerTimeout, [&] { return lb->taken >= mine; })) return TM_ERR_TRANSPORT;
   return rc;
 }
 

@@ -220,3 +220,19 @@ def test_leaver_and_joiner_in_two_processes(tmp_path):
         assert o["stats"]["rounds"] == 2 and o["stats"]["waves"] == 9 + 1 and o["stats"]["waves_again"] == 1
         assert o["checksums_ok"]
     assert rx["tensors_ok"] and rx["stats"]["bad_buckets"] == 1 and rx["stats"]["first_bad_bucket"] == 12
+
+
+def test_many_short_transfers_in_a_row(oracle_mod):
+    """Hundreds of waves of a few hundred bytes each: the hand-shakes between the two host threads (post,
+    match, take) follow one another as fast as they can, which is where a lost wake-up would show as
+    a partner time-out."""
+    specs = layouts.odd_specs(5, n_tensors=10)
+    state = layouts.materialize_adversarial(specs, "cuda", seed=5)
+    host = G.host_tensors(state)
+    _, exp_cks = oracle_mod.pack(host, 256)
+    for i in range(120):
+        target = layouts.blank_like(state)
+        tx, rx, _ = transfer.loopback_transfer(state.descs(), target.descs(), 256, 1 + i % 3, 1 + i % 4)
+        assert rx.stats["rounds"] == 1 and np.array_equal(G.u64(rx.checksums), exp_cks)
+        if i % 20 == 0:
+            _check_receiver(oracle_mod, state, target, tx, rx, 256)
