@@ -112,7 +112,7 @@ typedef struct tm_options {
   uint64_t small_bytes;        /* pieces below this share a work item, one warp per piece; default 8 KiB */
   uint64_t group_bytes;        /* byte budget of a shared item; default 64 KiB */
   uint64_t cksum_tile_bytes;   /* tile of the stand-alone checksum kernel; multiple of 256; default 256 KiB */
-  uint64_t wait_limit_ns;      /* bound of every device-side wait of the ring kernels; 1 .. 5e9; default 2e9 */
+  uint64_t wait_limit_ns;      /* bound of every device-side wait of the ring kernels; 1 .. 5e9; default 2e9.  Below 1024 (the timer's resolution) a wait that is not satisfied at once gives up at once: a diagnostic setting that makes launches end with TM_ERR_TIMEOUT and incomplete output */
   uint32_t group_max;          /* piece budget of a shared item; 1 .. 1024; default 64 */
   uint32_t ring_ctas_per_sm;   /* persistent blocks per SM of the ring kernels (96 KiB of shared memory each, 192 KiB in pack and unpack, where a second block does not fit); 1 .. 2; default 1 */
   uint32_t ctas_per_sm;        /* persistent blocks per SM of the checksum kernel; 1 .. 8; default 4 */

@@ -77,9 +77,24 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Waits for the phase with the given parity; gives up after limit_ns or when the block aborts.
+// Non-blocking probe of a barrier phase.
+__device__ __forceinline__ bool mbar_test(uint64_t* b, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(b)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+constexpr unsigned long long kTimerResolutionNs = 1024;   // limits below this cannot be measured with %globaltimer
+// Waits for the phase with the given parity; gives up after limit_ns or when the block aborts.  A
+// limit below the timer's resolution means "do not wait at all": the wait fails unless the phase has
+// already completed (used to drive the give-up paths of the kernels on purpose).
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag,
                                           unsigned long long limit_ns) {
+  if (mbar_test(b, parity)) return true;
+  if (limit_ns < kTimerResolutionNs) return false;
   if (mbar_try(b, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
