@@ -81,7 +81,7 @@ typedef enum tm_status {
   TM_OK           =  0,
   TM_ERR_ARG      = -1,  /* NULL pointer, zero count/size, odd nbytes, nbytes % elem_size != 0 */
   TM_ERR_ALIGN    = -2,  /* odd tensor address, bucket_bytes % 256 != 0, packed buffer not 256-byte aligned */
-  TM_ERR_CAPACITY = -3,  /* output, input or workspace buffer smaller than required */
+  TM_ERR_CAPACITY = -3,  /* output, input or workspace buffer smaller than required; work list too long to build; out of host memory */
   TM_ERR_OVERLAP  = -4,  /* a tensor overlaps the packed/output buffer, or two unpack targets overlap */
   TM_ERR_RANK     = -5,  /* D == 0 or r >= D */
   TM_ERR_DTYPE    = -6,  /* elem_size not in {2,4,8}, or mixed elem_size inside one shard plane */
