@@ -411,3 +411,62 @@ def test_results_do_not_depend_on_the_tuning_values(oracle_mod, opts):
         o = t.data_ptr() - target.arena.data_ptr()
         exp_arena[o:o + h.size] = h
     assert np.array_equal(target.arena.cpu().numpy(), exp_arena)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_layouts_through_the_fused_forms(oracle_mod, seed):
+    """Random small roles whose tensor sizes sit around the cuts that matter (16-byte vector, 2 KiB
+    bulk threshold, 8 KiB item threshold, 32 KiB stage, 256 KiB chunk), at random 2-byte-granular
+    addresses, with random bucket sizes, ranges, shard ranks and output alignments: the sender's fused
+    form (range plans through a slot) and the receiver's fused form must both equal the oracle."""
+    rng = np.random.default_rng(7000 + seed)
+    cuts = [16, 2048, 8192, 32768, 65536, 262144]
+    e = int(rng.choice([2, 4, 8]))
+    n = int(rng.integers(1, 7))
+    numels = []
+    for _ in range(n):
+        base = int(rng.choice(cuts)) * int(rng.integers(1, 4)) + int(rng.integers(-40, 41)) * 2
+        numels.append(max(1, base // e))
+    dtype = {2: torch.bfloat16, 4: torch.float32, 8: torch.int64}[e]
+    specs = [layouts.TensorSpec(f"t{k}", m, dtype, 1, k) for k, m in enumerate(numels)]
+    state = layouts.materialize_adversarial(specs, "cuda", seed=seed)
+    target = layouts.blank_like(state)
+    B = 256 * int(rng.choice([1, 3, 64, 1000, 4096]))
+    host = G.host_tensors(state)
+    exp_stream, exp_cks = oracle_mod.pack(host, B)
+    D = int(rng.integers(1, 6))
+    r = int(rng.integers(0, D))
+    expect = oracle_mod.shard(host, [h.size for h in host], e, r, D)
+    per = int(rng.integers(1, exp_cks.size + 1))
+    mis = 2 * int(rng.integers(0, 8))
+    tx_whole, tx_out = G.guarded(expect.size + 16)
+    rx_whole, rx_out = G.guarded(expect.size + 16)
+    tx_flat, rx_flat = tx_out[mis:mis + expect.size], rx_out[mis:mis + expect.size]
+    slot_whole, slot = G.guarded(per * B)
+    cks = torch.zeros(exp_cks.size, dtype=torch.int64, device="cuda")
+    got = torch.zeros(exp_cks.size, dtype=torch.int64, device="cuda")
+    stream_seen = torch.empty(exp_stream.size, dtype=torch.uint8, device="cuda")
+    first = 0
+    while first < exp_cks.size:
+        tx = RoleMover(state.descs(), B, first_bucket=first, n_buckets=per)
+        rx = RoleMover(target.descs(), B, first_bucket=first, n_buckets=per)
+        tx.attach_shards([(0, n)], r, D, outs=[tx_flat])
+        rx.attach_shards([(0, n)], r, D, outs=[rx_flat])
+        slot.fill_(0x3C)
+        tx.pack_emit(slot, cks[first:first + tx.n_buckets])
+        rx.unpack_emit(slot[:rx.total_bytes], got[first:first + rx.n_buckets])
+        torch.cuda.synchronize()
+        assert tx.status() == 0 and rx.status() == 0 and G.guards_intact(slot_whole, per * B)
+        stream_seen[tx.plan.stream_begin:tx.plan.stream_begin + tx.total_bytes] = slot[:tx.total_bytes]
+        first += per
+    ctx = (numels, e, B, per, r, D, mis)
+    assert np.array_equal(stream_seen.cpu().numpy(), exp_stream), ctx
+    assert np.array_equal(G.u64(cks), exp_cks) and np.array_equal(G.u64(got), exp_cks), ctx
+    assert np.array_equal(tx_flat.cpu().numpy(), expect) and np.array_equal(rx_flat.cpu().numpy(), expect), ctx
+    for whole in (tx_whole, rx_whole):
+        assert bool((whole[:G.GUARD + mis] == G.GUARD_BYTE).all()) and bool((whole[G.GUARD + mis + expect.size:] == G.GUARD_BYTE).all()), ctx
+    exp_arena = np.full(target.arena.numel(), 0xA5, dtype=np.uint8)
+    for t, h in zip(target.tensors, host):
+        o = t.data_ptr() - target.arena.data_ptr()
+        exp_arena[o:o + h.size] = h
+    assert np.array_equal(target.arena.cpu().numpy(), exp_arena), ctx
