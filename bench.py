@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 WORKLOADS = {"cfg0": 0, "cfg1": 1, "cfg2": 2, "cfg3": 3}
 # DRAM bytes (read + written) per algorithmic byte of the pack kernel, from the ncu capture summarised
 # in profiles/; None until the current kernel has been captured.
-RING_PACK_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9838
+RING_PACK_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9842
 TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum of ring_kernel<pack> captured on config 3 reduced to one "
-                "layer (1497.8 + 1449.0 MB for 2995.2 MB algorithmic), scaled by bytes moved; "
+                "layer (1497.9 + 1449.9 MB for 2995.2 MB algorithmic), scaled by bytes moved; "
                 "profiles/kernels_cfg3_1layer_ncu_counters.md")
 
 
